@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the compressed-CDC shuffle on B200.
+
+A step is one pass of the whole shuffle path (pre-combine + encode, then
+decode + cancel + reduce) over one batch of synthetic Map outputs that is
+already resident in device memory.  The workload is the distributed-SGD
+gradient shape (K=20, r=2, N=190, Q=20, 1.28 M floats per value, about 39 GB of
+intermediate values held across the 20 logical nodes), far larger than L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  ``value`` is intermediate-value GB/s: the bytes of Map
+output every node has to read for the shuffle, divided by the time of a step.
+With N > 1 (torchrun) every rank runs an independent job of the same shape
+(weak scaling, no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+from paper_1805_01993_b200.inputs import CONFIGS, DEFAULT_SEED, values_numpy, values_torch  # noqa: E402
+
+METRIC = "shuffle GB/s (combine+encode+decode+reduce)"
+UNIT = "GB/s"
+
+
+# ---------------------------------------------------------------- byte counts
+def algorithmic_bytes(K, r, N, Q, B, J=1, rounds=None):
+    """Bytes the method must move, node-faithful (each logical node's reads count;
+    pre-combined packets are recomputed, never stored)."""
+    from math import comb
+
+    length = (Q // K) * B
+    s = -(-length // r)
+    b = N // comb(K, r) if J == 1 else N // (r + 1)
+    rounds = comb(K, r + 1) if rounds is None else rounds
+    packets = rounds * (r + 1)                       # (round, receiver) pairs
+    enc_iv = packets * length * b * 4                # each packet built once, a segment per sender
+    dec_cancel = packets * (r - 1) * length * b * 4  # the other r-1 segments at each receiver
+    local = r * J * N * length * 4                   # own function's values
+    coded_w = packets * s * 4
+    coded_r = r * coded_w
+    out = J * Q * B * 4
+    return {
+        "iv_read": enc_iv + dec_cancel + local,
+        "encode_kernel": enc_iv + coded_w,
+        "decode_kernel": dec_cancel + local + coded_r + out,
+        "coded_write": coded_w,
+        "total": enc_iv + dec_cancel + local + coded_w + coded_r + out,
+    }
+
+
+# ---------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100", "-i", str(self.index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            text, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "power_w_max": max(power)}
+
+
+# ---------------------------------------------------------------- oracle legs
+def oracle_sample_shape(w, target_seconds):
+    """Same K, r, N, Q with the value shortened so one oracle pass takes about
+    ``target_seconds`` on one core; calibrated on a very short value first."""
+    from oracle.ccdc_oracle import Oracle
+
+    probe_B = w.r * 64
+    o = Oracle(w.K, w.r, w.N, w.Q, probe_B, w.dtype)
+    o.load_values(values_numpy(w.N, w.Q, probe_B, w.dtype, std=w.std))
+    t0 = time.perf_counter()
+    o.shuffle(); o.reduce()
+    per_elem = (time.perf_counter() - t0) / probe_B
+    B = int(target_seconds / per_elem) // (4 * w.r) * (4 * w.r)
+    return max(4 * w.r, min(B, w.B))
+
+
+def time_oracle(w, B):
+    """One oracle pass (shuffle + reduce; the copy of the Map outputs into the
+    node memories is not part of the shuffle and is not timed)."""
+    from oracle.ccdc_oracle import Oracle
+
+    o = Oracle(w.K, w.r, w.N, w.Q, B, w.dtype)
+    o.load_values(values_numpy(w.N, w.Q, B, w.dtype, std=w.std))
+    t0 = time.perf_counter()
+    o.shuffle(); o.reduce()
+    return time.perf_counter() - t0
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    total_budget = 150.0
+    B = oracle_sample_shape(w, total_budget / (args.steps + args.warmup))
+    for _ in range(args.warmup):
+        time_oracle(w, B)
+    t = [time_oracle(w, B) for _ in range(args.steps)]
+    per_step = sum(t) / len(t)
+    by = algorithmic_bytes(w.K, w.r, w.N, w.Q, B)
+    value = by["iv_read"] / per_step / 1e9
+    sample = f"{w.name} with B={B} of {w.B} elements per value (same K, r, N, Q), one pass per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+# ---------------------------------------------------------------- CUDA arm
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1805_01993_b200 import build as lib_build
+    from paper_1805_01993_b200 import ccdc
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        lib_build.build_library()
+    if world > 1:
+        dist.barrier()
+    ccdc.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    plan.upload()
+    part = plan.alloc_partitions(dev)
+    # every rank is an independent job of the same shape: its own seed
+    plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=DEFAULT_SEED + rank,
+                                                      std=w.std))
+    coded = plan.alloc(plan.coded_bytes, dev)
+    out = plan.alloc(plan.out_bytes, dev)
+    ws = plan.alloc(plan.workspace_bytes, dev)
+    by = algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B)
+    stream = torch.cuda.current_stream()
+
+    for _ in range(args.warmup):
+        plan.shuffle(part, coded, out, ws)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ccdc.num_kernel_launches()
+    barrier()
+    start.record(stream)
+    for i in range(args.steps):
+        ev[i][0].record(stream)
+        plan.encode_fused(part, coded)
+        ev[i][1].record(stream)
+        plan.decode_reduce(part, coded, out, ws)
+        ev[i][2].record(stream)
+    end.record(stream)
+    barrier()
+    launches = ccdc.num_kernel_launches() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    elapsed_ms = start.elapsed_time(end)
+    enc_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    dec_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = t.item() / args.steps
+    value = world * by["iv_read"] / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end through the host-buffer entry point ------------------
+    e2e = None
+    try:
+        import psutil
+
+        need = sum(plan.partition_bytes(k) for k in range(w.K)) + plan.out_bytes
+        if psutil.virtual_memory().available > 1.5 * need * min(world, 8) + (8 << 30):
+            host_part = [torch.empty(p.numel(), dtype=p.dtype, pin_memory=True) for p in part]
+            for h, p in zip(host_part, part):
+                h.copy_(p)
+            host_out = torch.empty(out.numel(), dtype=out.dtype, pin_memory=True)
+            e2e_steps = max(1, min(args.steps, 3))
+            plan.shuffle_host(host_part, host_out, part, coded, out, ws)      # warm-up
+            barrier()
+            s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s2.record(stream)
+            for _ in range(e2e_steps):
+                plan.shuffle_host(host_part, host_out, part, coded, out, ws)
+            e2.record(stream)
+            barrier()
+            t2 = torch.tensor([s2.elapsed_time(e2)], dtype=torch.float64, device=dev)
+            if world > 1:
+                dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+            e2e = {"value": world * by["iv_read"] / (t2.item() / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+                   "h2d_bytes_per_step": need - plan.out_bytes, "d2h_bytes_per_step": plan.out_bytes,
+                   "steps": e2e_steps, "ms_per_step": t2.item() / e2e_steps}
+            assert torch.equal(host_out, out.cpu())
+            del host_part
+        else:
+            e2e = {"value": None, "unit": UNIT, "skipped": "not enough free host memory for pinned copies"}
+    except Exception as exc:            # the device-resident number must still be reported
+        e2e = {"value": None, "unit": UNIT, "skipped": f"{type(exc).__name__}: {exc}"}
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peaks_file = ROOT / "MEASURED_PEAKS.json"
+    if peaks_file.exists():
+        peak, peak_kind = json.loads(peaks_file.read_text())["hbm_gbs"], "measured"
+    else:
+        peak, peak_kind = 6650.0, "fallback"
+    achieved = by["decode_kernel"] / (dec_ms * 1e-3) / 1e9
+    enc_achieved = by["encode_kernel"] / (enc_ms * 1e-3) / 1e9
+    traffic_file = ROOT / "profiles" / "traffic.json"
+    traffic = None
+    if traffic_file.exists():
+        traffic = json.loads(traffic_file.read_text()).get("decode_kernel_bytes_per_launch")
+
+    cpu = None
+    if world == 1:
+        Bs = oracle_sample_shape(w, 15.0)
+        secs = time_oracle(w, Bs)
+        bs = algorithmic_bytes(w.K, w.r, w.N, w.Q, Bs)
+        cpu = {"value": bs["iv_read"] / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{w.name} with B={Bs} of {w.B} elements per value (same K, r, N, Q), one pass, "
+                         f"{secs:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
+                   "l2": "inputs (38.9 GB) larger than L2, no flush", "jobs_per_gpu": 1,
+                   "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
+                   "algorithmic_bytes_per_step": by["total"],
+                   "hbm_frac_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9 / peak},
+        "roofline": {"bound": "hbm", "kernel": "k_decode_reduce", "achieved": achieved, "peak": peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                     "ms_per_launch": dec_ms,
+                     "other_kernels": {"k_gather(encode)": {"achieved": enc_achieved, "frac": enc_achieved / peak,
+                                                            "ms_per_launch": enc_ms}}},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="cfg4", choices=sorted(CONFIGS))
+    args = ap.parse_args()
+    w = CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,201 @@
+/*
+ * ccdc.h -- C ABI of the compressed coded distributed computing (compressed
+ * CDC) shuffle for one NVIDIA B200 (sm_100a).
+ *
+ * The method is that of Li, Maddah-Ali and Avestimehr, "Compressed Coded
+ * Distributed Computing": a MapReduce job with linear aggregation (Eq. (1)),
+ * N files placed on K nodes with computation load r = mu*K (Section IV-A),
+ * Q Reduce functions, Q/K per node (Section III).  In the Shuffle phase every
+ * node pre-combines, by summation over a batch of files, the intermediate
+ * values another node needs, XORs equal segments of r such packets into one
+ * coded multicast packet per (r+1)-subset, and every receiver cancels what it
+ * can rebuild from its own Map results (Section IV-B).
+ *
+ * Here the K nodes are logical: each node's Map results live in a partition of
+ * one GPU's memory, and a multicast is a write into a shared buffer that the r
+ * receivers read.  A kernel acting for node k dereferences node k's buffers
+ * and the shared coded buffer only.
+ *
+ * Conventions
+ *   - Every function returns CCDC_OK (0) or a negative ccdc_status; nothing
+ *     throws, aborts or traps.  Arguments are validated before any launch.
+ *   - The library owns only the plan (host tables and, after the first device
+ *     call or ccdc_plan_upload, their device copies on the device that was
+ *     current then).  The caller owns every data buffer and the stream.
+ *   - "device pointer array": a HOST array of K pointers to DEVICE memory,
+ *     entry k belonging to node k.  Data pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     All step functions are asynchronous on it; a step that follows another
+ *     on the same stream sees its results.
+ *   - Elements are 32 bits wide: int32 with wrapping addition or IEEE binary32.
+ *     XOR coding acts on the raw bit patterns in both cases.
+ *
+ * Layouts (element = 32-bit word; len = (Q/K)*B; s = ceil(len / r))
+ *   partition of node k   [local batch][file in batch][q = 0..Q-1][B]
+ *                         local batches = the batches whose label contains k,
+ *                         in ascending batch id; files ascending.
+ *   packets of node k     [local batch][outside node t, ascending][len]
+ *                         (stepwise API only)
+ *   coded buffer          [round][sender rank inside the round's subset][s_pad]
+ *                         s_pad = s rounded up to a multiple of 4 words; only
+ *                         the first s words of a row are multicast bits.
+ *   decoded of node k     [rounds that contain k, ascending][len]
+ *                         (stepwise API only)
+ *   out                   [job][q = 0..Q-1][B]; function q belongs to node
+ *                         q / (Q/K).
+ */
+#ifndef CCDC_H
+#define CCDC_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ccdc_plan_s ccdc_plan_t;     /* opaque; created and destroyed by the library */
+
+typedef enum { CCDC_I32 = 0, CCDC_F32 = 1 } ccdc_dtype_t;
+
+typedef enum {
+    CCDC_OK = 0,
+    CCDC_EINVAL = -1,   /* parameters outside the paper's setting, NULL or misaligned pointer */
+    CCDC_ENOMEM = -2,   /* host or device allocation of plan tables failed */
+    CCDC_ECUDA = -3,    /* a CUDA call or launch failed; see ccdc_last_cuda_error */
+    CCDC_ESIZE = -4,    /* a size exceeds what the entry point supports */
+    CCDC_ESTATE = -5    /* call not valid for this plan (e.g. ccdc_map on a plan without a Map) */
+} ccdc_status;
+
+#define CCDC_MAX_K 32   /* nodes; the subset tables grow as C(K, r+1) */
+
+/* ------------------------------------------------------------------ plan
+ * Section IV-A (file placement), Section III (function assignment S_k) and the
+ * multicast schedule of Section IV-B.
+ *
+ * ccdc_plan: ONE job over all K nodes.  The N files are cut into C(K,r)
+ * batches of b = N / C(K,r) consecutive files; batch p is labelled by the p-th
+ * size-r subset of {0..K-1} in lexicographic order and stored at those r
+ * nodes.  There is one multicast round per size-(r+1) subset S (lexicographic):
+ * member t of S receives the batch labelled S\{t}.  Node k reduces functions
+ * k*Q/K .. (k+1)*Q/K-1.
+ *   requires 2 <= K <= CCDC_MAX_K, 1 <= r <= K-1, K <= N, C(K,r) | N, K | Q,
+ *   B >= 1; otherwise CCDC_EINVAL and *out = NULL.
+ *
+ * ccdc_plan_jobs: the scheme as Section IV states it for J = C(K,r+1) jobs
+ * (gamma = 1).  Job j lives on the j-th size-(r+1) subset K_j; its N files are
+ * cut into r+1 batches labelled by the size-r subsets of K_j (lexicographic).
+ * Rounds, for each subset S = K_j in order: stage 1, then one stage-2 round
+ * per outside node i ascending, in which member t receives the batch labelled
+ * S\{t} of the job living on {i} U S\{t}.  Global file id = j*N + n; global
+ * function id = j*Q + q.   requires additionally (r+1) | N.
+ *
+ * Host only: no CUDA call is made.  Destroy with ccdc_plan_destroy. */
+int  ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
+int  ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
+void ccdc_plan_destroy(ccdc_plan_t *plan);
+
+/* Copies the schedule tables to the current device (cudaMalloc + cudaMemcpy,
+ * synchronous).  Optional: the first step call on a plan does it implicitly.
+ * After it no step function allocates.  CCDC_ENOMEM / CCDC_ECUDA on failure. */
+int  ccdc_plan_upload(ccdc_plan_t *plan);
+
+/* ---------------------------------------------------------------- queries
+ * All host side, valid for the plan's lifetime.  Index arguments out of range
+ * give CCDC_EINVAL (or 0 for the size queries). */
+long long ccdc_plan_num_jobs(const ccdc_plan_t *plan);        /* J */
+long long ccdc_plan_num_batches(const ccdc_plan_t *plan);     /* over all jobs */
+long long ccdc_plan_num_groups(const ccdc_plan_t *plan);      /* multicast rounds: C(K,r+1) per job batch set */
+long long ccdc_plan_files_per_batch(const ccdc_plan_t *plan); /* b */
+long long ccdc_plan_packet_elems(const ccdc_plan_t *plan);    /* len = (Q/K)*B */
+long long ccdc_plan_segment_elems(const ccdc_plan_t *plan);   /* s = ceil(len/r) */
+long long ccdc_plan_coded_row_elems(const ccdc_plan_t *plan); /* s_pad */
+/* exact number of bits multicast: rounds * (r+1) * 32 * s  (Definition 1 counts a broadcast once) */
+long long ccdc_plan_coded_bits(const ccdc_plan_t *plan);
+/* nodes_out[r]: ascending ids of the nodes storing global file n */
+int  ccdc_plan_batch_of_file(const ccdc_plan_t *plan, long long n, int *nodes_out);
+/* nodes_out[r] = label of batch p; *first_file = its first global file id; *job = its job */
+int  ccdc_plan_batch(const ccdc_plan_t *plan, long long p, int *nodes_out, long long *first_file, long long *job);
+/* members_out[r+1]: ascending node ids of round g */
+int  ccdc_plan_group(const ccdc_plan_t *plan, long long g, int *members_out);
+/* batches_out[r+1]: batch id whose packet member a of round g receives */
+int  ccdc_plan_group_batches(const ccdc_plan_t *plan, long long g, long long *batches_out);
+/* number of batches stored at node k, and their ids (ascending) into ids_out (may be NULL) */
+long long ccdc_plan_node_batches(const ccdc_plan_t *plan, int k, long long *ids_out);
+
+size_t ccdc_partition_bytes(const ccdc_plan_t *plan, int k);  /* node k's Map results */
+size_t ccdc_packets_bytes(const ccdc_plan_t *plan, int k);    /* stepwise API */
+size_t ccdc_decoded_bytes(const ccdc_plan_t *plan, int k);    /* stepwise API */
+size_t ccdc_coded_bytes(const ccdc_plan_t *plan);             /* shared multicast buffer */
+size_t ccdc_out_bytes(const ccdc_plan_t *plan);               /* J*Q*B*4 */
+size_t ccdc_workspace_bytes(const ccdc_plan_t *plan);         /* ccdc_shuffle scratch; may be 0 */
+
+/* ------------------------------------------------------------------ steps
+ * part, packets, decoded: device pointer arrays (see above). */
+
+/* Pre-combining (Section IV-B): packets[k][local batch][t] = concatenation over
+ * q in S_t of  sum_{n in batch} v_{q,n}, files added in ascending order
+ * starting from the first file's value. */
+int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packets, void *stream);
+
+/* Encoding (Section IV-B, message X_k): coded[round][a] = XOR over the other
+ * members t of the round of segment (label = sender) of the sender's packet
+ * for t; segments are s words, the last one zero extended. */
+int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void *stream);
+
+/* Decoding (Section IV-B): for every node k, round containing k and sender
+ * k' != k: coded packet XOR the r-1 segments labelled k' of k's own packets
+ * for the other members = segment labelled k' of the packet meant for k. */
+int ccdc_decode(ccdc_plan_t *plan, const void *const *packets, const void *coded,
+                void *const *decoded, void *stream);
+
+/* Reduce (Eq. (1), final reduction of Section IV): out[j][q] = sum over the
+ * batches of job j, ascending, of the local pre-combined value (batch stored at
+ * the node of q) or the decoded one. */
+int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *decoded,
+                void *out, void *stream);
+
+/* The four steps fused into two launches (plus a small deterministic final
+ * pass when the batch loop is split): pre-combining is recomputed inside the
+ * encode and inside the decode, decoded packets are never stored, every value
+ * a node needs is read from its partition once.
+ *
+ * ccdc_encode_fused: launch 1.  coded[round][a] straight from the sender's
+ *   partition (pre-combining of Section IV-B + message X_k).  Bit-identical to
+ *   ccdc_combine followed by ccdc_encode.
+ * ccdc_decode_reduce: launch 2.  For node k, each of its output words: over
+ *   the batches of the job in ascending order, the local pre-combined word, or
+ *   the coded word XOR the r-1 cancellable pre-combined words (decoding of
+ *   Section IV-B), accumulated as Eq. (1) demands.  workspace:
+ *   ccdc_workspace_bytes (may be NULL if that is 0); it is fully overwritten
+ *   before it is read.  int32 outputs are bit-identical to the stepwise path;
+ *   fp32 outputs are too when the workspace size is 0, and otherwise differ
+ *   from it only by the grouping of the per-batch terms.
+ * ccdc_shuffle: both, in order, on `stream`.
+ *   coded: ccdc_coded_bytes; out: ccdc_out_bytes. */
+int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, void *stream);
+int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
+                       void *workspace, void *stream);
+int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out,
+                 void *workspace, void *stream);
+
+/* ccdc_shuffle on Map results that live in HOST memory (Section III: the
+ * Shuffle phase starts from each node's local Map results and ends with the
+ * Reduce outputs at the nodes).  host_part: host array of K HOST pointers,
+ * node k's partition (ccdc_partition_bytes(k); pinned memory makes the copies
+ * asynchronous); host_out: HOST buffer of ccdc_out_bytes.  dev_part, dev_coded,
+ * dev_out, dev_workspace: device staging buffers of the usual sizes, owned by
+ * the caller.  Enqueues on `stream`: K host-to-device copies, the two
+ * launches, one device-to-host copy of the outputs; returns without waiting. */
+int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *host_out,
+                      void *const *dev_part, void *dev_coded, void *dev_out, void *dev_workspace,
+                      void *stream);
+
+/* ------------------------------------------------------------- diagnostics */
+const char *ccdc_strerror(int status);
+int ccdc_last_cuda_error(void);          /* cudaError_t of the last CCDC_ECUDA on this thread */
+int ccdc_num_kernel_launches(void);      /* kernels launched by this library so far (process wide) */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCDC_H */

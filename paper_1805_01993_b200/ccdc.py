@@ -1,0 +1,287 @@
+"""Python binding of the C-ABI library ``libccdc.so`` (declared in ``include/ccdc.h``).
+
+Argument marshalling only: every step of the shuffle runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  The function names are
+those of the C ABI; ``Plan`` wraps a ``ccdc_plan_t`` and offers the same calls as
+methods taking torch tensors.
+
+There is no fallback: if the shared library has not been built (see
+``paper_1805_01993_b200.build``) importing a symbol from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_LIB_PATH = Path(__file__).resolve().parent / "libccdc.so"
+_lib = None
+
+I32, F32 = 0, 1
+OK, EINVAL, ENOMEM, ECUDA, ESIZE, ESTATE = 0, -1, -2, -3, -4, -5
+MAX_K = 32
+
+_P, _I, _LL, _SZ = ctypes.c_void_p, ctypes.c_int, ctypes.c_longlong, ctypes.c_size_t
+_PP = ctypes.POINTER(ctypes.c_void_p)
+
+# name -> (restype, argtypes); mirrors include/ccdc.h
+SIGNATURES = {
+    "ccdc_plan": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
+    "ccdc_plan_jobs": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
+    "ccdc_plan_destroy": (None, [_P]),
+    "ccdc_plan_upload": (_I, [_P]),
+    "ccdc_plan_num_jobs": (_LL, [_P]),
+    "ccdc_plan_num_batches": (_LL, [_P]),
+    "ccdc_plan_num_groups": (_LL, [_P]),
+    "ccdc_plan_files_per_batch": (_LL, [_P]),
+    "ccdc_plan_packet_elems": (_LL, [_P]),
+    "ccdc_plan_segment_elems": (_LL, [_P]),
+    "ccdc_plan_coded_row_elems": (_LL, [_P]),
+    "ccdc_plan_coded_bits": (_LL, [_P]),
+    "ccdc_plan_batch_of_file": (_I, [_P, _LL, _P]),
+    "ccdc_plan_batch": (_I, [_P, _LL, _P, _P, _P]),
+    "ccdc_plan_group": (_I, [_P, _LL, _P]),
+    "ccdc_plan_group_batches": (_I, [_P, _LL, _P]),
+    "ccdc_plan_node_batches": (_LL, [_P, _I, _P]),
+    "ccdc_partition_bytes": (_SZ, [_P, _I]),
+    "ccdc_packets_bytes": (_SZ, [_P, _I]),
+    "ccdc_decoded_bytes": (_SZ, [_P, _I]),
+    "ccdc_coded_bytes": (_SZ, [_P]),
+    "ccdc_out_bytes": (_SZ, [_P]),
+    "ccdc_workspace_bytes": (_SZ, [_P]),
+    "ccdc_combine": (_I, [_P, _PP, _PP, _P]),
+    "ccdc_encode": (_I, [_P, _PP, _P, _P]),
+    "ccdc_decode": (_I, [_P, _PP, _P, _PP, _P]),
+    "ccdc_reduce": (_I, [_P, _PP, _PP, _P, _P]),
+    "ccdc_encode_fused": (_I, [_P, _PP, _P, _P]),
+    "ccdc_decode_reduce": (_I, [_P, _PP, _P, _P, _P, _P]),
+    "ccdc_shuffle": (_I, [_P, _PP, _P, _P, _P, _P]),
+    "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
+    "ccdc_strerror": (ctypes.c_char_p, [_I]),
+    "ccdc_last_cuda_error": (_I, []),
+    "ccdc_num_kernel_launches": (_I, []),
+}
+
+
+class CcdcError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().ccdc_strerror(status).decode()
+        if status == ECUDA:
+            msg += f" [cudaError {lib().ccdc_last_cuda_error()}]"
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+def lib():
+    """The loaded shared library; raises if it is missing (there is no other path)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise ImportError(f"{_LIB_PATH} not built: run `python -m paper_1805_01993_b200.build`")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = L
+    return _lib
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise CcdcError(status, where)
+
+
+def _ptr_array(tensors):
+    arr = (ctypes.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t.data_ptr() if t is not None and t.numel() > 0 else None
+    return arr
+
+
+def _stream_handle(stream):
+    import torch
+
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class Plan:
+    """``ccdc_plan`` / ``ccdc_plan_jobs`` plus the step calls on torch tensors."""
+
+    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False):
+        self.K, self.r, self.N, self.Q, self.B = K, r, N, Q, B
+        self.dtype = {"int32": I32, "float32": F32, I32: I32, F32: F32}[dtype]
+        self.jobs = jobs
+        h = ctypes.c_void_p()
+        fn = lib().ccdc_plan_jobs if jobs else lib().ccdc_plan
+        self._h = None
+        _check(fn(K, r, N, Q, B, self.dtype, ctypes.byref(h)), "ccdc_plan")
+        self._h = h
+        L = lib()
+        self.J = L.ccdc_plan_num_jobs(h)
+        self.num_batches = L.ccdc_plan_num_batches(h)
+        self.num_groups = L.ccdc_plan_num_groups(h)
+        self.files_per_batch = L.ccdc_plan_files_per_batch(h)
+        self.packet_elems = L.ccdc_plan_packet_elems(h)
+        self.segment_elems = L.ccdc_plan_segment_elems(h)
+        self.coded_row_elems = L.ccdc_plan_coded_row_elems(h)
+        self.coded_bits = L.ccdc_plan_coded_bits(h)
+
+    def __del__(self):
+        if getattr(self, "_h", None) and _lib is not None:
+            _lib.ccdc_plan_destroy(self._h)
+            self._h = None
+
+    # ---- queries --------------------------------------------------------
+    def batch_of_file(self, n):
+        out = (ctypes.c_int * self.r)()
+        _check(lib().ccdc_plan_batch_of_file(self._h, n, out), "ccdc_plan_batch_of_file")
+        return list(out)
+
+    def batch(self, p):
+        nodes = (ctypes.c_int * self.r)()
+        f0, job = ctypes.c_longlong(), ctypes.c_longlong()
+        _check(lib().ccdc_plan_batch(self._h, p, nodes, ctypes.byref(f0), ctypes.byref(job)), "ccdc_plan_batch")
+        return list(nodes), f0.value, job.value
+
+    def group(self, g):
+        out = (ctypes.c_int * (self.r + 1))()
+        _check(lib().ccdc_plan_group(self._h, g, out), "ccdc_plan_group")
+        return list(out)
+
+    def group_batches(self, g):
+        out = (ctypes.c_longlong * (self.r + 1))()
+        _check(lib().ccdc_plan_group_batches(self._h, g, out), "ccdc_plan_group_batches")
+        return list(out)
+
+    def node_batches(self, k):
+        n = lib().ccdc_plan_node_batches(self._h, k, None)
+        out = (ctypes.c_longlong * max(n, 1))()
+        lib().ccdc_plan_node_batches(self._h, k, out)
+        return list(out)[:n]
+
+    def partition_bytes(self, k):
+        return lib().ccdc_partition_bytes(self._h, k)
+
+    def packets_bytes(self, k):
+        return lib().ccdc_packets_bytes(self._h, k)
+
+    def decoded_bytes(self, k):
+        return lib().ccdc_decoded_bytes(self._h, k)
+
+    @property
+    def coded_bytes(self):
+        return lib().ccdc_coded_bytes(self._h)
+
+    @property
+    def out_bytes(self):
+        return lib().ccdc_out_bytes(self._h)
+
+    @property
+    def workspace_bytes(self):
+        return lib().ccdc_workspace_bytes(self._h)
+
+    def node_files(self, k):
+        """global file ids in the order of node k's partition rows."""
+        files = []
+        for p in self.node_batches(k):
+            _, f0, _ = self.batch(p)
+            files.extend(range(f0, f0 + self.files_per_batch))
+        return files
+
+    # ---- device buffers (torch is the allocator) --------------------------
+    @property
+    def torch_dtype(self):
+        import torch
+
+        return torch.int32 if self.dtype == I32 else torch.float32
+
+    def upload(self):
+        _check(lib().ccdc_plan_upload(self._h), "ccdc_plan_upload")
+
+    def alloc(self, nbytes, device="cuda"):
+        import torch
+
+        return torch.empty(max(nbytes // 4, 0), dtype=self.torch_dtype, device=device)
+
+    def alloc_partitions(self, device="cuda"):
+        return [self.alloc(self.partition_bytes(k), device) for k in range(self.K)]
+
+    def alloc_packets(self, device="cuda"):
+        return [self.alloc(self.packets_bytes(k), device) for k in range(self.K)]
+
+    def alloc_decoded(self, device="cuda"):
+        return [self.alloc(self.decoded_bytes(k), device) for k in range(self.K)]
+
+    def fill_partitions(self, part, values):
+        """Copies Map outputs ``values`` [J*N][Q][B] (tensor on any device) into the
+        node partitions: each node gets a replica of every file it stores."""
+        import torch
+
+        row = self.Q * self.B
+        flat = values.reshape(-1, row)
+        for k in range(self.K):
+            idx = torch.as_tensor(self.node_files(k), dtype=torch.long, device=flat.device)
+            if idx.numel():
+                part[k].view(-1, row).copy_(flat.index_select(0, idx), non_blocking=False)
+
+    def fill_partitions_streaming(self, part, file_iter, sample_index=None):
+        """Places files one at a time: ``file_iter`` yields ``(n, tensor [Q][B])`` on
+        the partitions' device; each is copied to the r nodes that store file n.
+        With ``sample_index`` (1-D long tensor of element positions) also returns
+        the sampled values ``[J*N][Q][len(sample_index)]`` on the host."""
+        import torch
+
+        row = self.Q * self.B
+        where = [{n: i for i, n in enumerate(self.node_files(k))} for k in range(self.K)]
+        sampled = None
+        if sample_index is not None:
+            sampled = torch.empty((self.J * self.N, self.Q, sample_index.numel()), dtype=self.torch_dtype)
+        for n, t in file_iter:
+            for k in self.batch_of_file(n):
+                i = where[k][n]
+                part[k][i * row:(i + 1) * row].copy_(t.reshape(-1))
+            if sampled is not None:
+                sampled[n] = t.index_select(1, sample_index).cpu()
+        return sampled
+
+    # ---- steps ------------------------------------------------------------
+    def combine(self, part, packets, stream=None):
+        _check(lib().ccdc_combine(self._h, _ptr_array(part), _ptr_array(packets), _stream_handle(stream)),
+               "ccdc_combine")
+
+    def encode(self, packets, coded, stream=None):
+        _check(lib().ccdc_encode(self._h, _ptr_array(packets), coded.data_ptr(), _stream_handle(stream)),
+               "ccdc_encode")
+
+    def decode(self, packets, coded, decoded, stream=None):
+        _check(lib().ccdc_decode(self._h, _ptr_array(packets), coded.data_ptr(), _ptr_array(decoded),
+                                 _stream_handle(stream)), "ccdc_decode")
+
+    def reduce(self, part, decoded, out, stream=None):
+        _check(lib().ccdc_reduce(self._h, _ptr_array(part), _ptr_array(decoded), out.data_ptr(),
+                                 _stream_handle(stream)), "ccdc_reduce")
+
+    def encode_fused(self, part, coded, stream=None):
+        _check(lib().ccdc_encode_fused(self._h, _ptr_array(part), coded.data_ptr(), _stream_handle(stream)),
+               "ccdc_encode_fused")
+
+    def decode_reduce(self, part, coded, out, workspace=None, stream=None):
+        ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None
+        _check(lib().ccdc_decode_reduce(self._h, _ptr_array(part), coded.data_ptr(), out.data_ptr(), ws,
+                                        _stream_handle(stream)), "ccdc_decode_reduce")
+
+    def shuffle_host(self, host_part, host_out, part, coded, out, workspace=None, stream=None):
+        """``host_part`` / ``host_out``: CPU tensors (pinned for asynchronous copies)."""
+        ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None
+        _check(lib().ccdc_shuffle_host(self._h, _ptr_array(host_part), host_out.data_ptr(), _ptr_array(part),
+                                       coded.data_ptr(), out.data_ptr(), ws, _stream_handle(stream)),
+               "ccdc_shuffle_host")
+
+    def shuffle(self, part, coded, out, workspace=None, stream=None):
+        ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None
+        _check(lib().ccdc_shuffle(self._h, _ptr_array(part), coded.data_ptr(), out.data_ptr(), ws,
+                                  _stream_handle(stream)), "ccdc_shuffle")
+
+
+def num_kernel_launches() -> int:
+    return lib().ccdc_num_kernel_launches()

@@ -1,0 +1,549 @@
+// CUDA kernels (sm_100a) and launch code of the compressed CDC shuffle.
+//
+// All steps are streaming: at most one add or XOR per 32-bit word moved, so
+// the kernels are organised around wide coalesced loads with many independent
+// loads in flight per thread, and tables of element offsets prepared by the
+// host planner.  A thread block that works for node k reads node k's buffers
+// and the shared coded buffer only.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <algorithm>
+#include <cstring>
+#include <type_traits>
+
+#include "ccdc_internal.h"
+
+namespace {
+
+constexpr int THREADS = CCDC_THREADS;
+constexpr int UNROLL = CCDC_UNROLL;
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<int> g_launches{0};
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = (int)e;
+    return CCDC_ECUDA;
+}
+
+// ---------------------------------------------------------------- vectors
+template <int VEC> struct WordVec;
+template <> struct WordVec<1> { using type = unsigned int; };
+template <> struct WordVec<2> { using type = uint2; };
+template <> struct WordVec<4> { using type = uint4; };
+
+template <int VEC> struct Words { uint32_t w[VEC]; };
+
+template <int VEC>
+__device__ __forceinline__ Words<VEC> load_words(const uint32_t *p) {
+    using V = typename WordVec<VEC>::type;
+    V v = __ldg(reinterpret_cast<const V *>(p));
+    Words<VEC> out;
+    memcpy(out.w, &v, sizeof(V));
+    return out;
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_words(uint32_t *p, const Words<VEC> &x) {
+    using V = typename WordVec<VEC>::type;
+    V v;
+    memcpy(&v, x.w, sizeof(V));
+    *reinterpret_cast<V *>(p) = v;
+}
+
+template <int VEC>
+__device__ __forceinline__ Words<VEC> zero_words() {
+    Words<VEC> z;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) z.w[i] = 0u;
+    return z;
+}
+
+// the aggregation of Eq. (1): int32 wrapping add, or IEEE binary32 add
+template <bool F32>
+__device__ __forceinline__ uint32_t add_word(uint32_t a, uint32_t b) {
+    if (F32) return __float_as_uint(__fadd_rn(__uint_as_float(a), __uint_as_float(b)));
+    return a + b;
+}
+
+template <int VEC, bool F32>
+__device__ __forceinline__ void add_into(Words<VEC> &a, const Words<VEC> &b) {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) a.w[i] = add_word<F32>(a.w[i], b.w[i]);
+}
+
+template <int VEC>
+__device__ __forceinline__ void xor_into(Words<VEC> &a, const Words<VEC> &b) {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) a.w[i] ^= b.w[i];
+}
+
+// sum over the b files of a batch, ascending, starting from the first file's
+// value (pre-combined value of Section IV-B); zero where the segment does not exist
+template <int VEC, bool F32>
+__device__ __forceinline__ Words<VEC> batch_sum(const uint32_t *src, long long off, long long j,
+                                                long long vl, int b, long long file_stride) {
+    if (j >= vl) return zero_words<VEC>();
+    const uint32_t *p = src + off + j;
+    Words<VEC> acc = load_words<VEC>(p);
+    for (int f = 1; f < b; ++f) {
+        p += file_stride;
+        add_into<VEC, F32>(acc, load_words<VEC>(p));
+    }
+    return acc;
+}
+
+// ---------------------------------------------------------------- gather
+// dst row = [coded row XOR] XOR over operands of the batch sums of a segment.
+// Serves pre-combining (1 operand), encoding (r operands) and the stepwise
+// decode (coded row and r-1 operands).
+struct GatherParams {
+    const uint32_t *src[CCDC_MAX_K];
+    uint32_t *dst[CCDC_MAX_K];
+    const uint32_t *coded_in;
+    const ccdc_row *rows;
+    const ccdc_ref *refs;
+    long long nrows;
+    long long tiles_per_row;
+    long long file_stride;
+    int na;
+    int b;
+};
+
+template <int VEC, bool F32>
+__global__ void __launch_bounds__(THREADS)
+k_gather(const __grid_constant__ GatherParams p) {
+    constexpr long long TILE = (long long)THREADS * VEC * UNROLL;
+    const long long item = blockIdx.x;
+    const long long row = item / p.tiles_per_row;
+    const long long tile = item - row * p.tiles_per_row;
+    if (row >= p.nrows) return;
+    const ccdc_row R = p.rows[row];
+    const long long j0 = tile * TILE + (long long)threadIdx.x * VEC;
+    if (tile * TILE >= R.n) return;
+    const uint32_t *src = p.src[R.src_node];
+    uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
+    const ccdc_ref *refs = p.refs + row * p.na;
+
+    Words<VEC> x[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const long long j = j0 + (long long)u * THREADS * VEC;
+        x[u] = (R.coded_off >= 0 && j < R.n) ? load_words<VEC>(p.coded_in + R.coded_off + j)
+                                             : zero_words<VEC>();
+    }
+    for (int a = 0; a < p.na; ++a) {
+        const ccdc_ref E = refs[a];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long j = j0 + (long long)u * THREADS * VEC;
+            if (j < R.n) xor_into<VEC>(x[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const long long j = j0 + (long long)u * THREADS * VEC;
+        if (j < R.n) store_words<VEC>(dst + j, x[u]);
+    }
+}
+
+// ------------------------------------------------------ fused decode + reduce
+// One block: node k (row of outputs), one segment i, one tile of it, one chunk
+// of the job's batches.  For each batch, ascending: the locally pre-combined
+// value if k stores the batch, else the coded word XOR the r-1 cancellable
+// pre-combined words (Section IV-B decoding), added to the accumulator
+// (Eq. (1)).  Decoded packets never reach memory.
+struct DecodeParams {
+    const uint32_t *part[CCDC_MAX_K];
+    const uint32_t *coded;
+    uint32_t *out;          // [out rows][len] when nchunk == 1
+    uint32_t *ws;           // [nchunk][out rows][len] otherwise
+    const ccdc_ref *terms;  // [out rows][r][nterm][TS]
+    long long nout;         // out rows = J*K
+    long long len, s;
+    long long file_stride;
+    long long tiles_per_seg;
+    long long nterm, terms_per_chunk;
+    int K, r, b, TS, nchunk;
+    int stage_terms;        // terms staged in shared memory at a time
+};
+
+template <int VEC, bool F32>
+__global__ void __launch_bounds__(THREADS)
+k_decode_reduce(const __grid_constant__ DecodeParams p) {
+    constexpr long long TILE = (long long)THREADS * VEC * UNROLL;
+    extern __shared__ ccdc_ref sh_terms[];
+
+    long long item = blockIdx.x;
+    const long long tile = item % p.tiles_per_seg; item /= p.tiles_per_seg;
+    const int i = (int)(item % p.r); item /= p.r;
+    const int chunk = (int)(item % p.nchunk);
+    const long long orow = item / p.nchunk;
+    if (orow >= p.nout) return;
+
+    const long long seglen = min(p.s, max(0LL, p.len - (long long)i * p.s));
+    if (tile * TILE >= seglen) return;
+    const int k = (int)(orow % p.K);
+    const uint32_t *src = p.part[k];
+    const long long j0 = tile * TILE + (long long)threadIdx.x * VEC;
+    const int r1 = p.r - 1;
+
+    const long long t_begin = (long long)chunk * p.terms_per_chunk;
+    const long long t_end = min(p.nterm, t_begin + p.terms_per_chunk);
+    const ccdc_ref *table = p.terms + ((orow * p.r + i) * p.nterm) * p.TS;
+
+    Words<VEC> acc[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) acc[u] = zero_words<VEC>();
+
+    for (long long t0 = t_begin; t0 < t_end; t0 += p.stage_terms) {
+        const int nt = (int)min((long long)p.stage_terms, t_end - t0);
+        __syncthreads();
+        for (int x = threadIdx.x; x < nt * p.TS; x += THREADS) sh_terms[x] = table[t0 * p.TS + x];
+        __syncthreads();
+        for (int t = 0; t < nt; ++t) {
+            const ccdc_ref *e = sh_terms + t * p.TS;
+            const long long coded_off = e[0].off;
+            Words<VEC> v[UNROLL];
+            if (coded_off < 0) {
+                const ccdc_ref E = e[1];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const long long j = j0 + (long long)u * THREADS * VEC;
+                    v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u) {
+                    const long long j = j0 + (long long)u * THREADS * VEC;
+                    v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
+                }
+                for (int c = 1; c <= r1; ++c) {
+                    const ccdc_ref E = e[c];
+#pragma unroll
+                    for (int u = 0; u < UNROLL; ++u) {
+                        const long long j = j0 + (long long)u * THREADS * VEC;
+                        if (j < seglen)
+                            xor_into<VEC>(v[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
+        }
+    }
+    uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) +
+                    orow * p.len + (long long)i * p.s;
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const long long j = j0 + (long long)u * THREADS * VEC;
+        if (j < seglen) store_words<VEC>(dst + j, acc[u]);
+    }
+}
+
+// final pass of the split batch loop: out = ((ws[0] + ws[1]) + ...) in chunk order
+template <bool F32>
+__global__ void __launch_bounds__(THREADS)
+k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, long long n, int nchunk) {
+    const long long e = (long long)blockIdx.x * THREADS + threadIdx.x;
+    if (e >= n) return;
+    uint32_t acc = ws[e];
+    for (int c = 1; c < nchunk; ++c) acc = add_word<F32>(acc, ws[(long long)c * n + e]);
+    out[e] = acc;
+}
+
+// ------------------------------------------------------ stepwise reduce
+// out row of node k = sum over the job's batches, ascending, of the local
+// pre-combined value or the decoded packet (Eq. (1)).
+struct ReduceParams {
+    const uint32_t *part[CCDC_MAX_K];
+    const uint32_t *decoded[CCDC_MAX_K];
+    uint32_t *out;
+    const ccdc_ref *terms;  // [out rows][nterm]
+    long long nout, len, nterm, file_stride, tiles_per_row;
+    int K, b;
+};
+
+template <int VEC, bool F32>
+__global__ void __launch_bounds__(THREADS)
+k_reduce(const __grid_constant__ ReduceParams p) {
+    constexpr long long TILE = (long long)THREADS * VEC;
+    const long long orow = blockIdx.x / p.tiles_per_row;
+    const long long tile = blockIdx.x - orow * p.tiles_per_row;
+    if (orow >= p.nout) return;
+    const long long j = tile * TILE + (long long)threadIdx.x * VEC;
+    if (j >= p.len) return;
+    const int k = (int)(orow % p.K);
+    const ccdc_ref *terms = p.terms + orow * p.nterm;
+    Words<VEC> acc = zero_words<VEC>();
+    for (long long t = 0; t < p.nterm; ++t) {
+        const ccdc_ref E = terms[t];
+        Words<VEC> v = E.vl == 0 ? batch_sum<VEC, F32>(p.part[k], E.off, j, p.len, p.b, p.file_stride)
+                                 : load_words<VEC>(p.decoded[k] + E.off + j);
+        add_into<VEC, F32>(acc, v);
+    }
+    store_words<VEC>(p.out + orow * p.len + j, acc);
+}
+
+// ---------------------------------------------------------------- launching
+template <typename F>
+int dispatch(const ccdc_plan_s &P, F &&f) {
+    const bool f32 = P.dtype == CCDC_F32;
+    switch (P.vec) {
+    case 4: return f32 ? f(std::integral_constant<int, 4>(), std::true_type()) : f(std::integral_constant<int, 4>(), std::false_type());
+    case 2: return f32 ? f(std::integral_constant<int, 2>(), std::true_type()) : f(std::integral_constant<int, 2>(), std::false_type());
+    default: return f32 ? f(std::integral_constant<int, 1>(), std::true_type()) : f(std::integral_constant<int, 1>(), std::false_type());
+    }
+}
+
+int check_launch() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? CCDC_OK : cuda_fail(e);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_ptr_array(const ccdc_plan_s &P, const void *const *a, bool (*nonempty)(const ccdc_plan_s &, int)) {
+    if (!a) return CCDC_EINVAL;
+    for (int k = 0; k < P.K; ++k) {
+        if (!nonempty(P, k)) continue;
+        if (!a[k] || !aligned16(a[k])) return CCDC_EINVAL;
+    }
+    return CCDC_OK;
+}
+
+bool has_part(const ccdc_plan_s &P, int k) { return P.nlocal[k] > 0; }
+bool has_decoded(const ccdc_plan_s &P, int k) { return P.node_nrounds[k] > 0; }
+
+int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *const *src, void *const *dst,
+                  void *dst_single, const void *coded_in, int b, long long file_stride, cudaStream_t st) {
+    if (T.rows.empty() || T.n_max == 0) return CCDC_OK;
+    GatherParams gp;
+    std::memset(&gp, 0, sizeof(gp));
+    for (int k = 0; k < P.K; ++k) {
+        gp.src[k] = static_cast<const uint32_t *>(src[k]);
+        gp.dst[k] = static_cast<uint32_t *>(dst_single ? dst_single : dst[k]);
+    }
+    gp.coded_in = static_cast<const uint32_t *>(coded_in);
+    gp.rows = T.d_rows; gp.refs = T.d_refs;
+    gp.nrows = (long long)T.rows.size();
+    gp.file_stride = file_stride; gp.na = T.na; gp.b = b;
+    return dispatch(P, [&](auto vec, auto f32) -> int {
+        constexpr int VEC = decltype(vec)::value;
+        constexpr bool F32 = decltype(f32)::value;
+        const long long tile = (long long)THREADS * VEC * UNROLL;
+        gp.tiles_per_row = (T.n_max + tile - 1) / tile;
+        const long long blocks = gp.nrows * gp.tiles_per_row;
+        if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
+        k_gather<VEC, F32><<<(unsigned)blocks, THREADS, 0, st>>>(gp);
+        return check_launch();
+    });
+}
+
+int ensure_device(ccdc_plan_s *plan) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (plan->device == dev) return CCDC_OK;
+    if (plan->device != -1) return CCDC_ESTATE;     // tables live on another device
+    return ccdc_plan_upload(plan);
+}
+
+}  // namespace
+
+void ccdc_internal_release_device(ccdc_plan_s *plan) {
+    if (plan->d_blob) {
+        int cur = -1;
+        cudaGetDevice(&cur);
+        if (cur != plan->device) cudaSetDevice(plan->device);
+        cudaFree(plan->d_blob);
+        if (cur != plan->device && cur >= 0) cudaSetDevice(cur);
+    }
+    plan->d_blob = nullptr;
+    plan->device = -1;
+}
+
+extern "C" {
+
+int ccdc_last_cuda_error(void) { return g_last_cuda_error; }
+int ccdc_num_kernel_launches(void) { return g_launches.load(); }
+
+int ccdc_plan_upload(ccdc_plan_t *plan) {
+    if (!plan) return CCDC_EINVAL;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (plan->device == dev) return CCDC_OK;
+    if (plan->device != -1) return CCDC_ESTATE;
+    struct Piece { const void *src; size_t bytes; const void **dst; };
+    ccdc_gather_table *tabs[4] = {&plan->enc_fused, &plan->cmb, &plan->enc_pk, &plan->dec_pk};
+    Piece pieces[10];
+    int np = 0;
+    for (ccdc_gather_table *T : tabs) {
+        pieces[np++] = {T->rows.data(), T->rows.size() * sizeof(ccdc_row), (const void **)&T->d_rows};
+        pieces[np++] = {T->refs.data(), T->refs.size() * sizeof(ccdc_ref), (const void **)&T->d_refs};
+    }
+    pieces[np++] = {plan->dec_terms.data(), plan->dec_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_dec_terms};
+    pieces[np++] = {plan->red_terms.data(), plan->red_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_red_terms};
+    size_t total = 0;
+    for (int i = 0; i < np; ++i) total += (pieces[i].bytes + 255) / 256 * 256;
+    void *blob = nullptr;
+    e = cudaMalloc(&blob, total ? total : 256);
+    if (e != cudaSuccess) { g_last_cuda_error = (int)e; return e == cudaErrorMemoryAllocation ? CCDC_ENOMEM : CCDC_ECUDA; }
+    size_t at = 0;
+    for (int i = 0; i < np; ++i) {
+        char *d = static_cast<char *>(blob) + at;
+        if (pieces[i].bytes) {
+            e = cudaMemcpy(d, pieces[i].src, pieces[i].bytes, cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) { cudaFree(blob); return cuda_fail(e); }
+        }
+        *pieces[i].dst = d;
+        at += (pieces[i].bytes + 255) / 256 * 256;
+    }
+    plan->d_blob = blob;
+    plan->device = dev;
+    return CCDC_OK;
+}
+
+int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packets, void *stream) {
+    if (!plan) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = check_ptr_array(*plan, (const void *const *)packets, has_part);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    return launch_gather(*plan, plan->cmb, part, packets, nullptr, nullptr, (int)plan->b, plan->row_elems,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void *stream) {
+    if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, packets, has_part);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    return launch_gather(*plan, plan->enc_pk, packets, nullptr, coded, nullptr, 1, 0,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int ccdc_decode(ccdc_plan_t *plan, const void *const *packets, const void *coded, void *const *decoded,
+                void *stream) {
+    if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, packets, has_part);
+    if (rc == CCDC_OK) rc = check_ptr_array(*plan, (const void *const *)decoded, has_decoded);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    return launch_gather(*plan, plan->dec_pk, packets, decoded, nullptr, coded, 1, 0,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *decoded, void *out, void *stream) {
+    if (!plan || !out || !aligned16(out)) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = check_ptr_array(*plan, decoded, has_decoded);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    const ccdc_plan_s &P = *plan;
+    ReduceParams rp;
+    std::memset(&rp, 0, sizeof(rp));
+    for (int k = 0; k < P.K; ++k) {
+        rp.part[k] = static_cast<const uint32_t *>(part[k]);
+        rp.decoded[k] = static_cast<const uint32_t *>(decoded[k]);
+    }
+    rp.out = static_cast<uint32_t *>(out);
+    rp.terms = P.d_red_terms;
+    rp.nout = P.J * P.K; rp.len = P.len; rp.nterm = P.nterm; rp.file_stride = P.row_elems;
+    rp.K = P.K; rp.b = (int)P.b;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    return dispatch(P, [&](auto vec, auto f32) -> int {
+        constexpr int VEC = decltype(vec)::value;
+        constexpr bool F32 = decltype(f32)::value;
+        const long long tile = (long long)THREADS * VEC;
+        rp.tiles_per_row = (P.len + tile - 1) / tile;
+        const long long blocks = rp.nout * rp.tiles_per_row;
+        if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
+        k_reduce<VEC, F32><<<(unsigned)blocks, THREADS, 0, st>>>(rp);
+        return check_launch();
+    });
+}
+
+int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, void *stream) {
+    if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    return launch_gather(*plan, plan->enc_fused, part, nullptr, coded, nullptr, (int)plan->b, plan->row_elems,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
+                       void *workspace, void *stream) {
+    if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
+    if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    const ccdc_plan_s &P = *plan;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    DecodeParams dp;
+    std::memset(&dp, 0, sizeof(dp));
+    for (int k = 0; k < P.K; ++k) dp.part[k] = static_cast<const uint32_t *>(part[k]);
+    dp.coded = static_cast<const uint32_t *>(coded);
+    dp.out = static_cast<uint32_t *>(out);
+    dp.ws = static_cast<uint32_t *>(workspace);
+    dp.terms = P.d_dec_terms;
+    dp.nout = P.J * P.K; dp.len = P.len; dp.s = P.s; dp.file_stride = P.row_elems;
+    dp.nterm = P.nterm; dp.terms_per_chunk = P.terms_per_chunk;
+    dp.K = P.K; dp.r = P.r; dp.b = (int)P.b; dp.TS = P.term_stride; dp.nchunk = P.nchunk;
+    const int stage_refs = 1024;                                    // 16 KiB of shared memory
+    dp.stage_terms = (int)std::max(1LL, std::min<long long>(stage_refs / P.term_stride, P.terms_per_chunk));
+    const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
+    return dispatch(P, [&](auto vec, auto f32) -> int {
+        constexpr int VEC = decltype(vec)::value;
+        constexpr bool F32 = decltype(f32)::value;
+        const long long tile = (long long)THREADS * VEC * UNROLL;
+        dp.tiles_per_seg = (P.s + tile - 1) / tile;
+        const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
+        if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
+        k_decode_reduce<VEC, F32><<<(unsigned)blocks, THREADS, smem, st>>>(dp);
+        int lrc = check_launch();
+        if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
+        const long long n = dp.nout * P.len;
+        k_sum_chunks<F32><<<(unsigned)((n + THREADS - 1) / THREADS), THREADS, 0, st>>>(dp.ws, dp.out, n, P.nchunk);
+        return check_launch();
+    });
+}
+
+int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out, void *workspace,
+                 void *stream) {
+    if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
+    if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
+    int rc = ccdc_encode_fused(plan, part, coded, stream);
+    if (rc != CCDC_OK) return rc;
+    return ccdc_decode_reduce(plan, part, coded, out, workspace, stream);
+}
+
+int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *host_out, void *const *dev_part,
+                      void *dev_coded, void *dev_out, void *dev_workspace, void *stream) {
+    if (!plan || !host_part || !host_out || !dev_part || !dev_coded || !dev_out) return CCDC_EINVAL;
+    if (!aligned16(dev_coded) || !aligned16(dev_out)) return CCDC_EINVAL;
+    if (plan->nchunk > 1 && (!dev_workspace || !aligned16(dev_workspace))) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, (const void *const *)dev_part, has_part);
+    if (rc != CCDC_OK) return rc;
+    for (int k = 0; k < plan->K; ++k)
+        if (has_part(*plan, k) && !host_part[k]) return CCDC_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int k = 0; k < plan->K; ++k) {
+        const size_t bytes = ccdc_partition_bytes(plan, k);
+        if (!bytes) continue;
+        cudaError_t e = cudaMemcpyAsync(dev_part[k], host_part[k], bytes, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    rc = ccdc_shuffle(plan, (const void *const *)dev_part, dev_coded, dev_out, dev_workspace, stream);
+    if (rc != CCDC_OK) return rc;
+    cudaError_t e = cudaMemcpyAsync(host_out, dev_out, ccdc_out_bytes(plan), cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess ? CCDC_OK : cuda_fail(e);
+}
+
+}  // extern "C"

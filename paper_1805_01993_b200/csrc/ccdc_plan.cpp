@@ -1,0 +1,487 @@
+// Host planner: file placement (Section IV-A), function assignment
+// (Section III, sets S_k) and the multicast schedule (Section IV-B) of the
+// compressed CDC scheme, flattened into the offset tables the kernels walk.
+// No CUDA call is made here.
+#include <algorithm>
+#include <climits>
+#include <cstring>
+#include <new>
+
+#include "ccdc_internal.h"
+
+namespace {
+
+// C(n, k), or -1 when it does not fit 62 bits
+long long choose(int n, int k) {
+    if (k < 0 || k > n) return 0;
+    k = std::min(k, n - k);
+    unsigned __int128 c = 1;
+    for (int i = 1; i <= k; ++i) {
+        c = c * (unsigned)(n - k + i) / (unsigned)i;
+        if (c > ((unsigned __int128)1 << 62)) return -1;
+    }
+    return (long long)c;
+}
+
+// lexicographic rank of the ascending m-subset c of {0..n-1}: the number of
+// m-subsets that precede it = those that agree on the first i entries and
+// carry a smaller value v at position i
+long long subset_rank(const int *c, int m, int n) {
+    long long rank = 0;
+    int lo = 0;
+    for (int i = 0; i < m; ++i) {
+        for (int v = lo; v < c[i]; ++v) rank += choose(n - 1 - v, m - 1 - i);
+        lo = c[i] + 1;
+    }
+    return rank;
+}
+
+// inverse of subset_rank
+void subset_unrank(long long rank, int m, int n, int *c) {
+    int v = 0;
+    for (int i = 0; i < m; ++i) {
+        for (;; ++v) {
+            long long cnt = choose(n - 1 - v, m - 1 - i);
+            if (rank < cnt) break;
+            rank -= cnt;
+        }
+        c[i] = v++;
+    }
+}
+
+int index_in(const int *set, int m, int x) {
+    for (int i = 0; i < m; ++i) if (set[i] == x) return i;
+    return -1;
+}
+
+long long seg_valid(const ccdc_plan_s &P, int i) {
+    long long rest = P.len - (long long)i * P.s;
+    return std::max(0LL, std::min(P.s, rest));
+}
+
+// operand reference; a segment that does not exist (vl = 0) is never
+// dereferenced and gets offset 0 so that every stored offset is in bounds
+ccdc_ref seg_ref(long long off, long long vl) { return vl > 0 ? ccdc_ref{off, vl} : ccdc_ref{0, 0}; }
+
+// first element of the packet row (batch p, first file, functions of node t) in node k's partition
+long long part_row(const ccdc_plan_s &P, int k, long long p, int t) {
+    return P.slot[(size_t)k * P.nbatch + p] * P.b * P.row_elems + (long long)t * P.len;
+}
+
+// index of packet (batch p, for node t) among node k's packets: [local batch][outside node ascending]
+long long packet_index(const ccdc_plan_s &P, int k, long long p, int t) {
+    const int *lab = &P.batch_nodes[(size_t)p * P.r];
+    int before = 0;                          // members of the label smaller than t
+    for (int i = 0; i < P.r; ++i) if (lab[i] < t) ++before;
+    return P.slot[(size_t)k * P.nbatch + p] * (P.K - P.r) + (t - before);
+}
+
+int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
+    if (K < 2 || K > CCDC_MAX_K) return CCDC_EINVAL;
+    if (r < 1 || r > K - 1) return CCDC_EINVAL;            // mu*K in {1..K-1}
+    if (N < K) return CCDC_EINVAL;                         // K <= N
+    if (Q < K || Q % K != 0) return CCDC_EINVAL;           // K | Q
+    if (B < 1) return CCDC_EINVAL;
+    if (dtype != CCDC_I32 && dtype != CCDC_F32) return CCDC_EINVAL;
+    if (N > (1LL << 40) || B > (1LL << 40) || Q > (1 << 24)) return CCDC_ESIZE;
+    return CCDC_OK;
+}
+
+// everything that follows from batches + rounds
+int finish(ccdc_plan_s &P) {
+    const int K = P.K, r = P.r;
+    // storage
+    P.slot.assign((size_t)K * P.nbatch, -1);
+    P.nlocal.assign(K, 0);
+    for (long long p = 0; p < P.nbatch; ++p)
+        for (int i = 0; i < r; ++i) {
+            int k = P.batch_nodes[(size_t)p * r + i];
+            P.slot[(size_t)k * P.nbatch + p] = P.nlocal[k]++;
+        }
+    // who receives which batch in which round; every (batch, outside node) exactly once
+    P.recv_round.assign((size_t)P.nbatch * K, -1);
+    P.node_round_index.assign((size_t)P.nround * (r + 1), 0);
+    P.node_nrounds.assign(K, 0);
+    for (long long g = 0; g < P.nround; ++g) {
+        const int *S = &P.round_group[(size_t)g * (r + 1)];
+        for (int a = 0; a <= r; ++a) {
+            long long p = P.round_batch[(size_t)g * (r + 1) + a];
+            if (p < 0 || p >= P.nbatch) return CCDC_EINVAL;
+            const int *lab = &P.batch_nodes[(size_t)p * r];
+            for (int x = 0, y = 0; x <= r; ++x) {          // label must be S without S[a]
+                if (x == a) continue;
+                if (lab[y++] != S[x]) return CCDC_EINVAL;
+            }
+            long long &slot = P.recv_round[(size_t)p * K + S[a]];
+            if (slot != -1) return CCDC_EINVAL;
+            slot = g;
+            P.node_round_index[(size_t)g * (r + 1) + a] = P.node_nrounds[S[a]]++;
+        }
+    }
+    for (long long p = 0; p < P.nbatch; ++p)
+        for (int k = 0; k < K; ++k) {
+            bool inside = index_in(&P.batch_nodes[(size_t)p * r], r, k) >= 0;
+            if (inside != (P.recv_round[(size_t)p * K + k] == -1)) return CCDC_EINVAL;
+        }
+
+    // vector width: every segment start and length must be a multiple of it
+    P.vec = (P.s % 4 == 0 && P.len % 4 == 0) ? 4 : (P.s % 2 == 0 && P.len % 2 == 0) ? 2 : 1;
+    P.term_stride = 1 + std::max(r - 1, 1);
+
+    const long long nrows = P.nround * (r + 1);
+    // ---- fused encode: coded row <- r partition segments of the sender
+    // ---- stepwise encode: the same from the sender's materialised packets
+    P.enc_fused.na = P.enc_pk.na = r;
+    P.enc_fused.n_max = P.enc_pk.n_max = P.s;
+    P.enc_fused.rows.resize(nrows); P.enc_fused.refs.resize((size_t)nrows * r);
+    P.enc_pk.rows.resize(nrows);    P.enc_pk.refs.resize((size_t)nrows * r);
+    for (long long g = 0; g < P.nround; ++g) {
+        const int *S = &P.round_group[(size_t)g * (r + 1)];
+        const long long *bat = &P.round_batch[(size_t)g * (r + 1)];
+        for (int as = 0; as <= r; ++as) {
+            const long long cr = g * (r + 1) + as;
+            const int ks = S[as];
+            ccdc_row row{ks, 0, cr * P.s_pad, P.s, -1};
+            P.enc_fused.rows[cr] = row;
+            P.enc_pk.rows[cr] = row;
+            int n = 0;
+            for (int a = 0; a <= r; ++a) {
+                if (a == as) continue;
+                const long long p = bat[a];
+                const int i = index_in(&P.batch_nodes[(size_t)p * r], r, ks);
+                const long long vl = seg_valid(P, i);
+                P.enc_fused.refs[(size_t)cr * r + n] = seg_ref(part_row(P, ks, p, S[a]) + (long long)i * P.s, vl);
+                P.enc_pk.refs[(size_t)cr * r + n] = seg_ref(packet_index(P, ks, p, S[a]) * P.len + (long long)i * P.s, vl);
+                ++n;
+            }
+        }
+    }
+    // ---- stepwise combine: packet <- sum over the batch's files
+    P.cmb.na = 1; P.cmb.n_max = P.len;
+    for (int k = 0; k < K; ++k)
+        for (long long p = 0; p < P.nbatch; ++p) {
+            if (P.slot[(size_t)k * P.nbatch + p] < 0) continue;
+            for (int t = 0; t < K; ++t) {
+                if (index_in(&P.batch_nodes[(size_t)p * r], r, t) >= 0) continue;
+                P.cmb.rows.push_back({k, k, packet_index(P, k, p, t) * P.len, P.len, -1});
+                P.cmb.refs.push_back({part_row(P, k, p, t), P.len});
+            }
+        }
+    // ---- stepwise decode: decoded segment <- coded XOR r-1 own packet segments
+    const int r1 = r - 1;
+    P.dec_pk.na = r1; P.dec_pk.n_max = P.s;
+    for (long long g = 0; g < P.nround; ++g) {
+        const int *S = &P.round_group[(size_t)g * (r + 1)];
+        const long long *bat = &P.round_batch[(size_t)g * (r + 1)];
+        for (int ak = 0; ak <= r; ++ak) {
+            const int k = S[ak];
+            const long long ridx = P.node_round_index[(size_t)g * (r + 1) + ak];
+            for (int as = 0; as <= r; ++as) {
+                if (as == ak) continue;
+                const int ks = S[as];
+                const int i0 = index_in(&P.batch_nodes[(size_t)bat[ak] * r], r, ks);
+                const long long n0 = seg_valid(P, i0);
+                P.dec_pk.rows.push_back({k, k, n0 > 0 ? ridx * P.len + (long long)i0 * P.s : 0, n0,
+                                         (g * (r + 1) + as) * P.s_pad});
+                for (int a = 0; a <= r; ++a) {
+                    if (a == ak || a == as) continue;
+                    const int i = index_in(&P.batch_nodes[(size_t)bat[a] * r], r, ks);
+                    P.dec_pk.refs.push_back(seg_ref(packet_index(P, k, bat[a], S[a]) * P.len + (long long)i * P.s,
+                                                    seg_valid(P, i)));
+                }
+            }
+        }
+    }
+    // ---- fused decode + reduce, and the stepwise reduce
+    const int TS = P.term_stride;
+    const long long nout = P.J * K;
+    P.dec_terms.assign((size_t)nout * r * P.nterm * TS, ccdc_ref{-1, 0});
+    P.red_terms.resize((size_t)nout * P.nterm);
+    for (long long j = 0; j < P.J; ++j)
+        for (int k = 0; k < K; ++k) {
+            const long long orow = j * K + k;
+            for (long long tt = 0; tt < P.nterm; ++tt) {
+                const long long p = P.job_batch0[j] + tt;
+                if (P.batch_job[p] != j) return CCDC_EINVAL;
+                const bool local = P.slot[(size_t)k * P.nbatch + p] >= 0;
+                const long long g = local ? -1 : P.recv_round[(size_t)p * K + k];
+                P.red_terms[(size_t)orow * P.nterm + tt] = local
+                    ? ccdc_ref{part_row(P, k, p, k), 0}
+                    : ccdc_ref{P.node_round_index[(size_t)g * (r + 1) +
+                                   index_in(&P.round_group[(size_t)g * (r + 1)], r + 1, k)] * P.len, 1};
+                for (int i = 0; i < r; ++i) {
+                    ccdc_ref *e = &P.dec_terms[(((size_t)orow * r + i) * P.nterm + tt) * TS];
+                    if (local) {
+                        e[0] = {-1, 0};
+                        e[1] = seg_ref(part_row(P, k, p, k) + (long long)i * P.s, seg_valid(P, i));
+                        continue;
+                    }
+                    const int *S = &P.round_group[(size_t)g * (r + 1)];
+                    const long long *bat = &P.round_batch[(size_t)g * (r + 1)];
+                    const int ak = index_in(S, r + 1, k);
+                    const int ks = P.batch_nodes[(size_t)p * r + i];    // sender whose label is segment i
+                    const int as = index_in(S, r + 1, ks);
+                    e[0] = {(g * (r + 1) + as) * P.s_pad, P.s};
+                    int n = 1;
+                    for (int a = 0; a <= r; ++a) {
+                        if (a == ak || a == as) continue;
+                        const int i2 = index_in(&P.batch_nodes[(size_t)bat[a] * r], r, ks);
+                        e[n++] = seg_ref(part_row(P, k, bat[a], S[a]) + (long long)i2 * P.s, seg_valid(P, i2));
+                    }
+                }
+            }
+        }
+
+    // ---- split of the batch loop of the fused decode: enough thread blocks to
+    // fill the GPU (148 SMs x 8 resident blocks) while a block still walks a
+    // fair number of batches
+    {
+        const long long tile = (long long)CCDC_THREADS * P.vec * CCDC_UNROLL;
+        const long long tiles_per_seg = (P.s + tile - 1) / tile;
+        const long long base = nout * r * tiles_per_seg;
+        long long want = (148LL * 8 + base - 1) / base;
+        long long cap = std::max(1LL, P.nterm / 8);
+        long long nch = std::max(1LL, std::min(want, cap));
+        P.terms_per_chunk = (P.nterm + nch - 1) / nch;
+        P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
+    }
+
+    // ---- every offset must stay inside its buffer
+    auto check_table = [&](const ccdc_gather_table &T, bool src_is_packets, bool dst_kind_coded,
+                           bool dst_is_packets, long long nf) -> bool {
+        for (size_t x = 0; x < T.rows.size(); ++x) {
+            const ccdc_row &R = T.rows[x];
+            if (R.src_node < 0 || R.src_node >= K || R.n < 0 || R.dst_off < 0) return false;
+            long long dst_cap = dst_kind_coded ? nrows * P.s_pad
+                              : dst_is_packets ? P.nlocal[R.dst_node] * (K - r) * P.len
+                                               : P.node_nrounds[R.dst_node] * P.len;
+            if (R.dst_off + R.n > dst_cap) return false;
+            if (R.coded_off >= 0 && R.coded_off + R.n > nrows * P.s_pad) return false;
+            long long src_cap = src_is_packets ? P.nlocal[R.src_node] * (K - r) * P.len
+                                               : P.nlocal[R.src_node] * P.b * P.row_elems;
+            for (int a = 0; a < T.na; ++a) {
+                const ccdc_ref &E = T.refs[x * T.na + a];
+                if (E.off < 0 || E.vl < 0 || E.vl > T.n_max) return false;
+                long long last = E.off + (nf - 1) * P.row_elems + std::min(E.vl, R.n);
+                if (last > src_cap) return false;
+            }
+        }
+        return true;
+    };
+    if (!check_table(P.enc_fused, false, true, false, P.b)) return CCDC_EINVAL;
+    if (!check_table(P.enc_pk, true, true, false, 1)) return CCDC_EINVAL;
+    if (!check_table(P.cmb, false, false, true, P.b)) return CCDC_EINVAL;
+    if (!check_table(P.dec_pk, true, false, false, 1)) return CCDC_EINVAL;
+    for (long long orow = 0; orow < nout; ++orow) {
+        const int k = (int)(orow % K);
+        const long long cap = P.nlocal[k] * P.b * P.row_elems;
+        for (size_t x = 0; x < (size_t)r * P.nterm; ++x) {
+            const ccdc_ref *e = &P.dec_terms[((size_t)orow * r * P.nterm + x) * TS];
+            const int nref = e[0].off < 0 ? 1 : r1;
+            if (e[0].off >= 0 && e[0].off + P.s > nrows * P.s_pad) return CCDC_EINVAL;
+            for (int c = 1; c <= nref; ++c)
+                if (e[c].off < 0 || e[c].off + (P.b - 1) * P.row_elems + e[c].vl > cap) return CCDC_EINVAL;
+        }
+    }
+    return CCDC_OK;
+}
+
+int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, bool jobs, ccdc_plan_t **out) {
+    if (!out) return CCDC_EINVAL;
+    *out = nullptr;
+    int rc = check_parameters(K, r, N, Q, B, (int)dtype);
+    if (rc != CCDC_OK) return rc;
+    const long long n_rsub = choose(K, r), n_r1sub = choose(K, r + 1);
+    if (n_rsub <= 0 || n_r1sub <= 0 || n_r1sub > (1LL << 24)) return CCDC_ESIZE;
+    if (!jobs && N % n_rsub != 0) return CCDC_EINVAL;       // batches of equal size
+    if (jobs && N % (r + 1) != 0) return CCDC_EINVAL;
+    try {
+        ccdc_plan_s *pp = new ccdc_plan_s();
+        ccdc_plan_s &P = *pp;
+        P.K = K; P.r = r; P.N = N; P.Q = Q; P.B = B; P.dtype = (int)dtype; P.jobs_mode = jobs;
+        P.len = (long long)(Q / K) * B;
+        P.s = (P.len + r - 1) / r;
+        P.s_pad = (P.s + 3) / 4 * 4;
+        P.row_elems = (long long)Q * B;
+        int c[CCDC_MAX_K + 1], rest[CCDC_MAX_K + 1];
+        if (!jobs) {
+            P.J = 1; P.b = N / n_rsub; P.nbatch = n_rsub; P.nround = n_r1sub; P.nterm = n_rsub;
+            P.job_batch0.assign(1, 0);
+            P.batch_nodes.resize((size_t)P.nbatch * r);
+            P.batch_file0.resize(P.nbatch); P.batch_job.assign(P.nbatch, 0);
+            for (long long p = 0; p < P.nbatch; ++p) {
+                subset_unrank(p, r, K, &P.batch_nodes[(size_t)p * r]);
+                P.batch_file0[p] = p * P.b;
+            }
+            P.round_group.resize((size_t)P.nround * (r + 1));
+            P.round_batch.resize((size_t)P.nround * (r + 1));
+            for (long long g = 0; g < P.nround; ++g) {
+                subset_unrank(g, r + 1, K, c);
+                std::memcpy(&P.round_group[(size_t)g * (r + 1)], c, sizeof(int) * (r + 1));
+                for (int a = 0; a <= r; ++a) {
+                    for (int x = 0, y = 0; x <= r; ++x) if (x != a) rest[y++] = c[x];
+                    P.round_batch[(size_t)g * (r + 1) + a] = subset_rank(rest, r, K);
+                }
+            }
+        } else {
+            P.J = n_r1sub; P.b = N / (r + 1); P.nbatch = P.J * (r + 1); P.nround = P.J * (K - r);
+            P.nterm = r + 1;
+            P.job_batch0.resize(P.J);
+            P.batch_nodes.resize((size_t)P.nbatch * r);
+            P.batch_file0.resize(P.nbatch); P.batch_job.resize(P.nbatch);
+            // the a-th size-r subset of an (r+1)-set in lexicographic order
+            // omits its (r-a)-th member
+            for (long long j = 0; j < P.J; ++j) {
+                subset_unrank(j, r + 1, K, c);
+                P.job_batch0[j] = j * (r + 1);
+                for (int a = 0; a <= r; ++a) {
+                    const long long p = j * (r + 1) + a;
+                    for (int x = 0, y = 0; x <= r; ++x) if (x != r - a) P.batch_nodes[(size_t)p * r + y++] = c[x];
+                    P.batch_job[p] = j;
+                    P.batch_file0[p] = j * N + a * P.b;
+                }
+            }
+            P.round_group.resize((size_t)P.nround * (r + 1));
+            P.round_batch.resize((size_t)P.nround * (r + 1));
+            long long g = 0;
+            for (long long j = 0; j < P.J; ++j) {
+                subset_unrank(j, r + 1, K, c);
+                // stage 1: member a receives job j's batch that omits it
+                std::memcpy(&P.round_group[(size_t)g * (r + 1)], c, sizeof(int) * (r + 1));
+                for (int a = 0; a <= r; ++a) P.round_batch[(size_t)g * (r + 1) + a] = j * (r + 1) + (r - a);
+                ++g;
+                // stage 2: one round per outside node i
+                for (int i = 0; i < K; ++i) {
+                    if (index_in(c, r + 1, i) >= 0) continue;
+                    std::memcpy(&P.round_group[(size_t)g * (r + 1)], c, sizeof(int) * (r + 1));
+                    for (int a = 0; a <= r; ++a) {
+                        // home of the job = {i} U S\{S[a]}, ascending; m = position of i in it
+                        int m = 0, y = 0;
+                        bool placed = false;
+                        for (int x = 0; x <= r; ++x) {
+                            if (x == a) continue;
+                            if (!placed && i < c[x]) { m = y; rest[y++] = i; placed = true; }
+                            rest[y++] = c[x];
+                        }
+                        if (!placed) { m = y; rest[y++] = i; }
+                        const long long jt = subset_rank(rest, r + 1, K);
+                        P.round_batch[(size_t)g * (r + 1) + a] = jt * (r + 1) + (r - m);
+                    }
+                    ++g;
+                }
+            }
+            if (g != P.nround) { delete pp; return CCDC_EINVAL; }
+        }
+        rc = finish(P);
+        if (rc != CCDC_OK) { delete pp; return rc; }
+        *out = pp;
+        return CCDC_OK;
+    } catch (const std::bad_alloc &) {
+        return CCDC_ENOMEM;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
+    return make_plan(K, r, N, Q, B, dtype, false, out);
+}
+
+int ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
+    return make_plan(K, r, N, Q, B, dtype, true, out);
+}
+
+void ccdc_plan_destroy(ccdc_plan_t *plan) {
+    if (!plan) return;
+    ccdc_internal_release_device(plan);
+    delete plan;
+}
+
+long long ccdc_plan_num_jobs(const ccdc_plan_t *p) { return p ? p->J : 0; }
+long long ccdc_plan_num_batches(const ccdc_plan_t *p) { return p ? p->nbatch : 0; }
+long long ccdc_plan_num_groups(const ccdc_plan_t *p) { return p ? p->nround : 0; }
+long long ccdc_plan_files_per_batch(const ccdc_plan_t *p) { return p ? p->b : 0; }
+long long ccdc_plan_packet_elems(const ccdc_plan_t *p) { return p ? p->len : 0; }
+long long ccdc_plan_segment_elems(const ccdc_plan_t *p) { return p ? p->s : 0; }
+long long ccdc_plan_coded_row_elems(const ccdc_plan_t *p) { return p ? p->s_pad : 0; }
+long long ccdc_plan_coded_bits(const ccdc_plan_t *p) { return p ? p->nround * (p->r + 1) * 32 * p->s : 0; }
+
+int ccdc_plan_batch_of_file(const ccdc_plan_t *p, long long n, int *nodes_out) {
+    if (!p || !nodes_out || n < 0 || n >= p->J * p->N) return CCDC_EINVAL;
+    const long long j = n / p->N, a = (n % p->N) / p->b;
+    const long long b = p->job_batch0[j] + a;
+    std::memcpy(nodes_out, &p->batch_nodes[(size_t)b * p->r], sizeof(int) * p->r);
+    return CCDC_OK;
+}
+
+int ccdc_plan_batch(const ccdc_plan_t *p, long long b, int *nodes_out, long long *first_file, long long *job) {
+    if (!p || b < 0 || b >= p->nbatch) return CCDC_EINVAL;
+    if (nodes_out) std::memcpy(nodes_out, &p->batch_nodes[(size_t)b * p->r], sizeof(int) * p->r);
+    if (first_file) *first_file = p->batch_file0[b];
+    if (job) *job = p->batch_job[b];
+    return CCDC_OK;
+}
+
+int ccdc_plan_group(const ccdc_plan_t *p, long long g, int *members_out) {
+    if (!p || !members_out || g < 0 || g >= p->nround) return CCDC_EINVAL;
+    std::memcpy(members_out, &p->round_group[(size_t)g * (p->r + 1)], sizeof(int) * (p->r + 1));
+    return CCDC_OK;
+}
+
+int ccdc_plan_group_batches(const ccdc_plan_t *p, long long g, long long *batches_out) {
+    if (!p || !batches_out || g < 0 || g >= p->nround) return CCDC_EINVAL;
+    std::memcpy(batches_out, &p->round_batch[(size_t)g * (p->r + 1)], sizeof(long long) * (p->r + 1));
+    return CCDC_OK;
+}
+
+long long ccdc_plan_node_batches(const ccdc_plan_t *p, int k, long long *ids_out) {
+    if (!p || k < 0 || k >= p->K) return 0;
+    if (ids_out) {
+        long long n = 0;
+        for (long long b = 0; b < p->nbatch; ++b)
+            if (p->slot[(size_t)k * p->nbatch + b] >= 0) ids_out[n++] = b;
+    }
+    return p->nlocal[k];
+}
+
+size_t ccdc_partition_bytes(const ccdc_plan_t *p, int k) {
+    if (!p || k < 0 || k >= p->K) return 0;
+    return (size_t)(p->nlocal[k] * p->b * p->row_elems) * 4;
+}
+
+size_t ccdc_packets_bytes(const ccdc_plan_t *p, int k) {
+    if (!p || k < 0 || k >= p->K) return 0;
+    return (size_t)(p->nlocal[k] * (p->K - p->r) * p->len) * 4;
+}
+
+size_t ccdc_decoded_bytes(const ccdc_plan_t *p, int k) {
+    if (!p || k < 0 || k >= p->K) return 0;
+    return (size_t)(p->node_nrounds[k] * p->len) * 4;
+}
+
+size_t ccdc_coded_bytes(const ccdc_plan_t *p) {
+    return p ? (size_t)(p->nround * (p->r + 1) * p->s_pad) * 4 : 0;
+}
+
+size_t ccdc_out_bytes(const ccdc_plan_t *p) { return p ? (size_t)(p->J * p->row_elems) * 4 : 0; }
+
+size_t ccdc_workspace_bytes(const ccdc_plan_t *p) {
+    if (!p || p->nchunk <= 1) return 0;
+    return (size_t)p->nchunk * (size_t)(p->J * p->row_elems) * 4;
+}
+
+const char *ccdc_strerror(int status) {
+    switch (status) {
+    case CCDC_OK: return "ok";
+    case CCDC_EINVAL: return "invalid argument (parameters outside the scheme's setting, NULL or misaligned pointer)";
+    case CCDC_ENOMEM: return "out of memory";
+    case CCDC_ECUDA: return "CUDA error (see ccdc_last_cuda_error)";
+    case CCDC_ESIZE: return "size not supported by this entry point";
+    case CCDC_ESTATE: return "call not valid for this plan";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,274 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI.
+
+Same seeded inputs on both sides.  int32: every packet, coded word, decoded word
+and output bit-exact.  fp32: coded packets bit-exact (the pre-combining order is
+fixed: files ascending, starting from the first file's value); outputs within
+1e-5 * sum_n |v_{q,n}| element-wise, the tolerance the method's evaluation
+states, since the fused path may add the per-batch terms in another grouping.
+"""
+import numpy as np
+import pytest
+
+from oracle.ccdc_oracle import Oracle
+from paper_1805_01993_b200.inputs import CONFIGS, values_numpy, values_torch
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+FP32_RTOL = 1e-5
+CANARY = 0x5A5A5A5A
+
+
+@pytest.fixture(scope="module")
+def ccdc():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_1805_01993_b200 import build, ccdc as mod
+
+    build.build_library()
+    mod.lib()
+    return mod
+
+
+def guarded(n_words, dtype, pad=64):
+    """tensor of n words with canary words on both sides; returns (whole, view)."""
+    whole = torch.full((n_words + 2 * pad,), CANARY, dtype=torch.int32, device="cuda")
+    return whole, whole[pad:pad + n_words].view(dtype)
+
+
+def canaries_intact(whole, n_words, pad=64):
+    w = whole.cpu().numpy().view(np.uint32)
+    return bool((w[:pad] == CANARY).all() and (w[pad + n_words:] == CANARY).all())
+
+
+def bits(t):
+    return t.detach().cpu().contiguous().numpy().view(np.uint32)
+
+
+def assert_outputs(out_gpu, o, dtype):
+    ref = o.reduce()
+    got = out_gpu.cpu().numpy().reshape(ref.shape)
+    if dtype == "int32":
+        assert np.array_equal(got, ref)
+        assert np.array_equal(got, o.direct())
+        return
+    s64, a64 = o.direct()
+    err = np.abs(got.astype(np.float64) - ref.astype(np.float64))
+    assert np.all(err <= FP32_RTOL * a64 + 1e-30), float((err / (a64 + 1e-30)).max())
+    assert np.all(np.abs(got - s64) <= FP32_RTOL * a64 + 1e-30)
+
+
+def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0):
+    plan = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+    o = Oracle(K, r, N, Q, B, dtype, mode="paper" if jobs else "single")
+    v = values_numpy(plan.J * N, Q, B, dtype, seed=seed, std=std)
+    o.load_values(v)
+    o.shuffle()
+    tdt = plan.torch_dtype
+    part = plan.alloc_partitions()
+    plan.fill_partitions(part, torch.from_numpy(v).cuda())
+    s, sp, L = plan.segment_elems, plan.coded_row_elems, plan.packet_elems
+    rows = plan.num_groups * (r + 1)
+    ref_coded = o.coded().reshape(rows, s)
+
+    # ---- stepwise path -------------------------------------------------
+    packets = plan.alloc_packets()
+    decoded = plan.alloc_decoded()
+    coded_w, coded = guarded(rows * sp, tdt)
+    out_w, out = guarded(plan.J * Q * B, tdt)
+    plan.combine(part, packets)
+    plan.encode(packets, coded)
+    plan.decode(packets, coded, decoded)
+    plan.reduce(part, decoded, out)
+    torch.cuda.synchronize()
+    for k in range(K):
+        assert np.array_equal(bits(packets[k]).reshape(-1, L), o.packets(k)), f"packets of node {k}"
+        assert np.array_equal(bits(decoded[k]).reshape(-1, L), o.decoded(k)), f"decoded of node {k}"
+    assert np.array_equal(bits(coded).reshape(rows, sp)[:, :s], ref_coded)
+    assert canaries_intact(coded_w, rows * sp) and canaries_intact(out_w, plan.J * Q * B)
+    assert_outputs(out, o, dtype)
+    # the stepwise reduce adds the batches in the oracle's order: same bits
+    assert np.array_equal(bits(out).reshape(-1, B), o.reduce().view(np.uint32))
+
+    # ---- fused path ------------------------------------------------------
+    coded_w2, coded2 = guarded(rows * sp, tdt)
+    out_w2, out2 = guarded(plan.J * Q * B, tdt)
+    ws_words = plan.workspace_bytes // 4
+    ws_w, ws = guarded(ws_words, tdt)
+    plan.shuffle(part, coded2, out2, ws if ws_words else None)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(coded2).reshape(rows, sp)[:, :s], ref_coded)
+    assert canaries_intact(coded_w2, rows * sp) and canaries_intact(out_w2, plan.J * Q * B)
+    assert canaries_intact(ws_w, ws_words)
+    assert_outputs(out2, o, dtype)
+    if ws_words == 0:
+        assert np.array_equal(bits(out2).reshape(-1, B), o.reduce().view(np.uint32))
+    assert plan.coded_bits == o.coded_bits
+    return plan
+
+
+# K, r, N, Q, B: r = 1, r = K-1, several files per batch, Q/K > 1, r does not
+# divide the packet, B < r, vector widths 1 / 2 / 4, several tiles + ragged tail
+SHAPES = [
+    (3, 2, 6, 3, 8),
+    (3, 1, 3, 3, 5),
+    (4, 2, 12, 4, 6),
+    (4, 3, 8, 4, 9),
+    (4, 1, 8, 8, 3),
+    (5, 2, 20, 5, 7),
+    (5, 3, 10, 10, 5),
+    (5, 4, 5, 5, 2),
+    (6, 3, 40, 6, 4),
+    (6, 2, 15, 12, 3),
+    (4, 2, 12, 4, 2 * (3 * 2048 + 20)),     # vec 4, 4 tiles per segment, ragged tail
+    (5, 3, 20, 5, 3 * (2 * 1024 + 6)),      # vec 2
+    (5, 3, 10, 5, 3 * 2049 + 1),            # vec 1, r does not divide B
+    (6, 5, 12, 6, 7001),                    # r = K-1, one round
+    (7, 3, 35, 14, 1000),                   # Q/K = 2
+]
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", SHAPES)
+def test_single_job_matches_oracle(ccdc, K, r, N, Q, B, dtype):
+    run_case(ccdc, K, r, N, Q, B, dtype, seed=K * 10 + r)
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", [(4, 2, 6, 4, 8), (5, 2, 9, 5, 37), (5, 3, 8, 10, 6), (6, 1, 6, 6, 5),
+                                       (6, 4, 10, 6, 4100)])
+def test_jobs_plan_matches_oracle(ccdc, K, r, N, Q, B, dtype):
+    """The scheme as stated for J = C(K, r+1) jobs (stages 1 and 2)."""
+    run_case(ccdc, K, r, N, Q, B, dtype, jobs=True, seed=3)
+
+
+def test_cfg1_full(ccdc):
+    w = CONFIGS["cfg1"]
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    assert plan.coded_bits == 49_152
+
+
+def test_cfg2_full(ccdc):
+    w = CONFIGS["cfg2"]
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    assert plan.coded_bits == 36_718_080 and plan.workspace_bytes > 0
+
+
+def test_cfg3_short_values(ccdc):
+    w = CONFIGS["cfg3"].scaled(512)
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    assert plan.workspace_bytes > 0
+
+
+def test_cfg4_short_values(ccdc):
+    w = CONFIGS["cfg4"].scaled(6000)
+    run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype, std=w.std)
+
+
+def test_cfg5_shuffle_shape(ccdc):
+    w = CONFIGS["cfg5"]
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    assert plan.coded_bits == 3_064_320
+
+
+def test_special_float_patterns_survive_coding(ccdc):
+    """-0.0, infinities and NaN payloads are carried bit for bit when b = 1."""
+    K, r, N, Q, B = 4, 2, 6, 4, 8
+    v = values_numpy(N, Q, B, "float32", seed=2)
+    v.view(np.uint32)[0, 3, 0] = 0x80000000
+    v.view(np.uint32)[1, 2, 1] = 0x7F800000
+    v.view(np.uint32)[2, 0, 2] = 0x7FC12345
+    plan = ccdc.Plan(K, r, N, Q, B, "float32")
+    o = Oracle(K, r, N, Q, B, "float32")
+    o.load_values(v)
+    o.shuffle()
+    part = plan.alloc_partitions()
+    plan.fill_partitions(part, torch.from_numpy(v).cuda())
+    coded = plan.alloc(plan.coded_bytes)
+    out = plan.alloc(plan.out_bytes)
+    plan.shuffle(part, coded, out, None)
+    packets, decoded = plan.alloc_packets(), plan.alloc_decoded()
+    plan.combine(part, packets)
+    plan.decode(packets, coded, decoded)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(coded).reshape(-1, plan.coded_row_elems)[:, :plan.segment_elems],
+                          o.coded().reshape(-1, plan.segment_elems))
+    for k in range(K):
+        assert np.array_equal(bits(decoded[k]).reshape(-1, B), o.decoded(k))
+
+
+def test_bad_arguments_are_refused(ccdc):
+    plan = ccdc.Plan(4, 2, 12, 4, 64, "int32")
+    part = plan.alloc_partitions()
+    coded = plan.alloc(plan.coded_bytes)
+    out = plan.alloc(plan.out_bytes)
+    before = ccdc.num_kernel_launches()
+    with pytest.raises(ccdc.CcdcError) as e:
+        plan.shuffle(part[:3] + [None], coded, out, None)
+    assert e.value.status == ccdc.EINVAL
+    with pytest.raises(ccdc.CcdcError):
+        plan.shuffle(part, coded[1:], out, None)            # misaligned
+    bigplan = ccdc.Plan(10, 3, 480, 10, 64, "int32")
+    assert bigplan.workspace_bytes > 0
+    bp = bigplan.alloc_partitions()
+    with pytest.raises(ccdc.CcdcError):
+        bigplan.shuffle(bp, bigplan.alloc(bigplan.coded_bytes), bigplan.alloc(bigplan.out_bytes), None)
+    assert ccdc.num_kernel_launches() == before
+    plan.shuffle(part, coded, out, None)
+    torch.cuda.synchronize()
+    assert ccdc.num_kernel_launches() == before + 2
+
+
+def sampled_full_size_check(ccdc, w, offsets_per_segment=48, seed=5):
+    """Full-size run in the benchmark's launch configuration, compared with the
+    oracle on a sub-problem: the same element offsets inside every segment form
+    an exact instance of the scheme with a shorter value (every step acts
+    element-wise along a segment), so the oracle can produce those coded words
+    and outputs one by one.  Requires r | B and Q = K."""
+    assert w.Q == w.K and w.B % w.r == 0
+    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    s = plan.segment_elems
+    rng = np.random.default_rng(seed)
+    tile = 256 * 4 * 2
+    fixed = [0, 1, 3, s - 1, s - 4, min(tile - 1, s - 1), min(tile, s - 1), s // 2]
+    offs = np.unique(np.concatenate([np.array(fixed), rng.integers(0, s, offsets_per_segment)]))
+    m = len(offs)
+    index = np.concatenate([i * s + offs for i in range(w.r)])
+    idx_t = torch.from_numpy(index).cuda()
+
+    part = plan.alloc_partitions()
+    sampled = plan.fill_partitions_streaming(
+        part, values_torch(w.N, w.Q, w.B, w.dtype, "cuda", seed=seed, std=w.std), idx_t)
+    coded = plan.alloc(plan.coded_bytes)
+    out = plan.alloc(plan.out_bytes)
+    ws = plan.alloc(plan.workspace_bytes) if plan.workspace_bytes else None
+    plan.shuffle(part, coded, out, ws)
+    torch.cuda.synchronize()
+
+    o = Oracle(w.K, w.r, w.N, w.Q, w.r * m, w.dtype)
+    o.load_values(sampled.numpy())
+    o.shuffle()
+    assert o.s == m
+    rows = plan.num_groups * (w.r + 1)
+    got_coded = coded.view(rows, plan.coded_row_elems).index_select(1, torch.from_numpy(offs).cuda())
+    assert np.array_equal(bits(got_coded), o.coded().reshape(rows, m))
+    got_out = out.view(w.Q, w.B).index_select(1, idx_t).cpu().numpy()
+    ref = o.reduce()
+    s64, a64 = o.direct()
+    err = np.abs(got_out.astype(np.float64) - ref.astype(np.float64))
+    assert np.all(err <= FP32_RTOL * a64 + 1e-30)
+    assert np.all(np.abs(got_out - s64) <= FP32_RTOL * a64 + 1e-30)
+    del part, coded, ws
+    return plan
+
+
+def test_cfg3_full_size_sampled(ccdc):
+    sampled_full_size_check(ccdc, CONFIGS["cfg3"])
+
+
+def test_cfg4_full_size_sampled(ccdc):
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60 * 2**30:
+        pytest.fail("cfg4 needs about 50 GB of device memory")
+    sampled_full_size_check(ccdc, CONFIGS["cfg4"], offsets_per_segment=24)

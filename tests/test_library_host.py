@@ -1,0 +1,118 @@
+"""Host-side checks of the C-ABI library: it loads, exports what the header
+declares, refuses what the paper's setting excludes, and its placement and
+multicast schedule agree with the oracle's (written independently)."""
+import ctypes
+import re
+from itertools import combinations
+from math import comb
+from pathlib import Path
+
+import pytest
+
+from oracle.ccdc_oracle import Oracle
+from paper_1805_01993_b200 import build as ccdc_build
+from paper_1805_01993_b200 import ccdc
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    ccdc_build.build_library()
+
+
+def declared_functions():
+    text = (ROOT / "include" / "ccdc.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ccdc_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_functions()
+    assert len(names) >= 25
+    handle = ctypes.CDLL(str(ccdc_build.LIB))
+    for name in names:
+        assert hasattr(handle, name), f"{name} declared in ccdc.h but not exported"
+    assert sorted(ccdc.SIGNATURES) == names, "Python binding and header disagree"
+
+
+def test_invalid_parameters():
+    bad = [(1, 1, 4, 1, 4), (4, 0, 12, 4, 8), (4, 4, 12, 4, 8), (4, 2, 3, 4, 8), (4, 2, 13, 4, 8),
+           (4, 2, 12, 6, 8), (4, 2, 12, 4, 0), (33, 2, 528, 33, 4)]
+    for args in bad:
+        with pytest.raises(ccdc.CcdcError) as e:
+            ccdc.Plan(*args, "int32")
+        assert e.value.status == ccdc.EINVAL
+    with pytest.raises(ccdc.CcdcError):
+        ccdc.Plan(4, 2, 7, 4, 8, "int32", jobs=True)
+    with pytest.raises(ccdc.CcdcError) as e:
+        ccdc.Plan(32, 15, comb(32, 15), 32, 8, "int32")       # schedule too large
+    assert e.value.status == ccdc.ESIZE
+    assert b"invalid" in ccdc.lib().ccdc_strerror(ccdc.EINVAL)
+    assert ccdc.lib().ccdc_plan_num_groups(None) == 0
+
+
+SHAPES = [(3, 2, 6, 3, 8), (4, 2, 12, 4, 6), (4, 1, 8, 8, 3), (5, 3, 10, 10, 5), (5, 4, 5, 5, 2),
+          (6, 3, 40, 6, 4), (7, 2, 21, 7, 9), (10, 3, 480, 10, 16)]
+
+
+@pytest.mark.parametrize("K,r,N,Q,B", SHAPES)
+def test_single_job_plan_matches_oracle_plan(K, r, N, Q, B):
+    p = ccdc.Plan(K, r, N, Q, B, "float32")
+    o = Oracle(K, r, N, Q, B, "float32")
+    assert (p.J, p.num_batches, p.num_groups, p.files_per_batch) == (1, o.nbatch, o.nround, o.b)
+    assert (p.packet_elems, p.segment_elems) == (o.len, o.s)
+    assert p.coded_row_elems % 4 == 0 and 0 <= p.coded_row_elems - o.s < 4
+    for b in range(o.nbatch):
+        nodes, f0, job = p.batch(b)
+        assert nodes == o.batch_nodes(b) and job == 0 and list(range(f0, f0 + o.b)) == o.batch_files(b)
+        for n in o.batch_files(b):
+            assert p.batch_of_file(n) == nodes
+    for g in range(o.nround):
+        assert p.group(g) == o.round_group(g) and p.group_batches(g) == o.round_batches(g)
+    assert p.coded_bits == comb(K, r + 1) * (r + 1) * 32 * o.s
+    for k in range(K):
+        assert p.partition_bytes(k) == o.node_num_files(k) * Q * B * 4
+        assert p.node_batches(k) == [b for b in range(o.nbatch) if k in o.batch_nodes(b)]
+        assert p.packets_bytes(k) == o.node_num_batches(k) * (K - r) * o.len * 4
+        assert p.decoded_bytes(k) == comb(K - 1, r) * o.len * 4
+    assert p.coded_bytes == o.nround * (r + 1) * p.coded_row_elems * 4
+    assert p.out_bytes == Q * B * 4
+
+
+@pytest.mark.parametrize("K,r,N", [(4, 2, 6), (5, 2, 9), (5, 3, 8), (6, 1, 6), (6, 4, 10)])
+def test_jobs_plan_matches_oracle_plan(K, r, N):
+    Q, B = K, 6
+    p = ccdc.Plan(K, r, N, Q, B, "int32", jobs=True)
+    o = Oracle(K, r, N, Q, B, "int32", mode="paper")
+    assert (p.J, p.num_batches, p.num_groups, p.files_per_batch) == (o.J, o.nbatch, o.nround, o.b)
+    for b in range(o.nbatch):
+        nodes, f0, job = p.batch(b)
+        assert nodes == o.batch_nodes(b) and job == o.batch_job(b) and f0 == o.batch_files(b)[0]
+    for g in range(o.nround):
+        assert p.group(g) == o.round_group(g) and p.group_batches(g) == o.round_batches(g)
+    # Theorem 1, from the library's own bit count (r | B here or padded: compare to s)
+    assert p.coded_bits == o.nround * (r + 1) * 32 * o.s
+    assert p.out_bytes == o.J * Q * B * 4
+
+
+def test_expected_bits_of_the_five_workloads():
+    expect = {(4, 2, 12, 4, 256): 49_152, (10, 3, 480, 10, 4096): 36_718_080,
+              (16, 4, 1820, 16, 16384): 2_862_612_480, (20, 2, 190, 20, 1_280_000): 70_041_600_000,
+              (8, 3, 112, 8, 1024): 3_064_320}
+    for shape, bits in expect.items():
+        assert ccdc.Plan(*shape, "float32").coded_bits == bits
+
+
+def test_storage_and_replication():
+    K, r, N, Q, B = 6, 3, 40, 6, 4
+    p = ccdc.Plan(K, r, N, Q, B, "int32")
+    seen = {}
+    for k in range(K):
+        files = p.node_files(k)
+        assert len(files) * K == r * N
+        for n in files:
+            seen.setdefault(n, []).append(k)
+    assert sorted(seen) == list(range(N))
+    assert all(len(v) == r and v == p.batch_of_file(n) for n, v in seen.items())
+    assert [p.batch(b)[0] for b in range(p.num_batches)] == [list(c) for c in combinations(range(K), r)]
