@@ -190,6 +190,31 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
                       void *const *dev_part, void *dev_coded, void *dev_out, void *dev_workspace,
                       void *stream);
 
+/* Allocation-free variant of ccdc_decode_reduce (the paper has no counterpart:
+ * this is a property of the library, not a step of the scheme).
+ *
+ * For callers that cannot allocate device memory where they shuffle -- code in
+ * a region where cudaMalloc is forbidden or would stall the device, or a
+ * program whose memory was handed out in full at start-up.  The scratch of the
+ * split batch loop is a fixed array of ccdc_static_scratch_bytes() (16 MiB) of
+ * device memory inside the library image; every GPU that loads the library
+ * holds it until the process exits.  The caller still passes inputs and
+ * outputs; results are identical to ccdc_decode_reduce.
+ *   - makes no cudaMalloc / cudaFree / allocating library call.  The plan's
+ *     tables must already be on the current device (ccdc_plan_upload, done
+ *     earlier by code that may allocate); otherwise CCDC_ESTATE.
+ *   - CCDC_ESIZE if ccdc_workspace_bytes(plan) exceeds the array.
+ *   - the first call on a device looks up the array's device address (once per
+ *     device, with that device current); make that first call before starting
+ *     any stream capture.
+ *   - all calls on a device share the array and it keeps the previous call's
+ *     contents; the kernels overwrite every word they later read, so nothing
+ *     needs clearing, but two calls whose kernels overlap on the GPU (different
+ *     streams, different plans or threads) race on it: serialise them. */
+size_t ccdc_static_scratch_bytes(void);
+int ccdc_decode_reduce_static(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
+                              void *stream);
+
 /* ------------------------------------------------------------- diagnostics */
 const char *ccdc_strerror(int status);
 int ccdc_last_cuda_error(void);          /* cudaError_t of the last CCDC_ECUDA on this thread */

@@ -55,6 +55,8 @@ SIGNATURES = {
     "ccdc_encode_fused": (_I, [_P, _PP, _P, _P]),
     "ccdc_decode_reduce": (_I, [_P, _PP, _P, _P, _P, _P]),
     "ccdc_shuffle": (_I, [_P, _PP, _P, _P, _P, _P]),
+    "ccdc_static_scratch_bytes": (_SZ, []),
+    "ccdc_decode_reduce_static": (_I, [_P, _PP, _P, _P, _P]),
     "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
     "ccdc_strerror": (ctypes.c_char_p, [_I]),
     "ccdc_last_cuda_error": (_I, []),
@@ -276,6 +278,11 @@ class Plan:
         _check(lib().ccdc_shuffle_host(self._h, _ptr_array(host_part), host_out.data_ptr(), _ptr_array(part),
                                        coded.data_ptr(), out.data_ptr(), ws, _stream_handle(stream)),
                "ccdc_shuffle_host")
+
+    def decode_reduce_static(self, part, coded, out, stream=None):
+        """``ccdc_decode_reduce`` with the library's built-in scratch: no allocation."""
+        _check(lib().ccdc_decode_reduce_static(self._h, _ptr_array(part), coded.data_ptr(), out.data_ptr(),
+                                               _stream_handle(stream)), "ccdc_decode_reduce_static")
 
     def shuffle(self, part, coded, out, workspace=None, stream=None):
         ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None

@@ -547,3 +547,61 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------
+// Allocation-free variant of ccdc_decode_reduce.
+//
+// Some callers cannot allocate device memory at the point where they shuffle:
+// code that runs inside a region where cudaMalloc is forbidden or would
+// synchronise the device (a latency-critical loop, a callback, a host thread
+// that must not touch the allocator), or a host program whose memory budget
+// was handed out in full at start-up.  For them the scratch of the split batch
+// loop lives in the library image itself: a fixed array in device global
+// memory that every GPU loading the library holds until the process exits.
+//
+// In host code the array's name is only a handle for the runtime, not a device
+// address, so the address is looked up with cudaGetSymbolAddress, once per
+// device with that device current, and that pointer is what the kernels get.
+constexpr size_t CCDC_STATIC_SCRATCH_BYTES = 16u << 20;     // 16 MiB
+static __device__ __align__(256) unsigned int g_static_scratch[CCDC_STATIC_SCRATCH_BYTES / 4];
+
+namespace {
+constexpr int MAX_DEVICES = 64;
+std::atomic<void *> g_static_scratch_ptr[MAX_DEVICES];
+
+// device address of the scratch array on the current device (set-up on first use)
+int static_scratch_address(void **out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= MAX_DEVICES) return CCDC_ESIZE;
+    void *p = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e);
+        g_static_scratch_ptr[dev].store(p, std::memory_order_release);
+    }
+    *out = p;
+    return CCDC_OK;
+}
+}  // namespace
+
+extern "C" {
+
+size_t ccdc_static_scratch_bytes(void) { return CCDC_STATIC_SCRATCH_BYTES; }
+
+int ccdc_decode_reduce_static(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
+                              void *stream) {
+    if (!plan) return CCDC_EINVAL;
+    if (ccdc_workspace_bytes(plan) > CCDC_STATIC_SCRATCH_BYTES) return CCDC_ESIZE;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (plan->device != dev) return CCDC_ESTATE;     // tables not uploaded here: uploading would allocate
+    void *scratch = nullptr;
+    int rc = static_scratch_address(&scratch);
+    if (rc != CCDC_OK) return rc;
+    return ccdc_decode_reduce(plan, part, coded, out, scratch, stream);
+}
+
+}  // extern "C"
