@@ -235,6 +235,8 @@ def run_ours(args, w):
     # ---- end to end through the host-buffer entry point ------------------
     e2e = None
     try:
+        if args.skip_e2e:
+            raise RuntimeError("--skip-e2e")
         import psutil
 
         need = sum(plan.partition_bytes(k) for k in range(w.K)) + plan.out_bytes
@@ -284,7 +286,7 @@ def run_ours(args, w):
         traffic = json.loads(traffic_file.read_text()).get("decode_kernel_bytes_per_launch")
 
     cpu = None
-    if world == 1:
+    if world == 1 and not args.skip_cpu_baseline:
         Bs = oracle_sample_shape(w, 15.0)
         secs = time_oracle(w, Bs)
         bs = algorithmic_bytes(w.K, w.r, w.N, w.Q, Bs)
@@ -297,7 +299,7 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
-                   "l2": "inputs (38.9 GB) larger than L2, no flush", "jobs_per_gpu": 1,
+                   "l2": f"inputs ({sum(plan.partition_bytes(k) for k in range(w.K)) / 1e9:.1f} GB) larger than L2, no flush", "jobs_per_gpu": 1,
                    "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
                    "algorithmic_bytes_per_step": by["total"],
                    "hbm_frac_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9 / peak},
@@ -321,8 +323,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="cfg4", choices=sorted(CONFIGS))
+    ap.add_argument("--value-elems", type=int, default=0,
+                    help="shorten every value to this many elements (profiling captures on a small case)")
+    ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg")
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave out the oracle timing leg")
     args = ap.parse_args()
     w = CONFIGS[args.workload]
+    if args.value_elems:
+        w = w.scaled(args.value_elems)
     if args.impl == "reference":
         run_reference(args, w)
     else:

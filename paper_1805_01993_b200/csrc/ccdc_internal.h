@@ -8,8 +8,14 @@
 
 // launch shape shared by the planner (which sizes the split of the fused
 // decode from it) and the kernels
-constexpr int CCDC_THREADS = 256;    // threads per block
-constexpr int CCDC_UNROLL = 2;       // vectors per thread per tile
+#ifndef CCDC_THREADS_PER_BLOCK
+#define CCDC_THREADS_PER_BLOCK 256
+#endif
+#ifndef CCDC_VECTORS_PER_THREAD
+#define CCDC_VECTORS_PER_THREAD 2
+#endif
+constexpr int CCDC_THREADS = CCDC_THREADS_PER_BLOCK;   // threads per block
+constexpr int CCDC_UNROLL = CCDC_VECTORS_PER_THREAD;   // vectors per thread per tile
 
 // One operand of a gathered segment: element offset into the owning node's
 // buffer (segment offset included) and the number of leading elements of the

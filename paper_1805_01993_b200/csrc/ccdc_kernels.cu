@@ -106,7 +106,8 @@ struct GatherParams {
     const ccdc_row *rows;
     const ccdc_ref *refs;
     long long nrows;
-    long long tiles_per_row;
+    long long spans_per_row;
+    long long span_elems;       // elements of a row one block covers (a multiple of the tile)
     long long file_stride;
     int na;
     int b;
@@ -116,36 +117,42 @@ template <int VEC, bool F32>
 __global__ void __launch_bounds__(THREADS)
 k_gather(const __grid_constant__ GatherParams p) {
     constexpr long long TILE = (long long)THREADS * VEC * UNROLL;
+    __shared__ ccdc_ref sh_refs[CCDC_MAX_K];
     const long long item = blockIdx.x;
-    const long long row = item / p.tiles_per_row;
-    const long long tile = item - row * p.tiles_per_row;
+    const long long row = item / p.spans_per_row;
+    const long long span = item - row * p.spans_per_row;
     if (row >= p.nrows) return;
     const ccdc_row R = p.rows[row];
-    const long long j0 = tile * TILE + (long long)threadIdx.x * VEC;
-    if (tile * TILE >= R.n) return;
+    const long long begin = span * p.span_elems;
+    const long long end = min(R.n, begin + p.span_elems);
+    if (begin >= end) return;
+    if (threadIdx.x < p.na) sh_refs[threadIdx.x] = p.refs[row * p.na + threadIdx.x];
+    __syncthreads();
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
-    const ccdc_ref *refs = p.refs + row * p.na;
 
-    Words<VEC> x[UNROLL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        const long long j = j0 + (long long)u * THREADS * VEC;
-        x[u] = (R.coded_off >= 0 && j < R.n) ? load_words<VEC>(p.coded_in + R.coded_off + j)
-                                             : zero_words<VEC>();
-    }
-    for (int a = 0; a < p.na; ++a) {
-        const ccdc_ref E = refs[a];
+    for (long long base = begin; base < end; base += TILE) {
+        const long long j0 = base + (long long)threadIdx.x * VEC;
+        Words<VEC> x[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const long long j = j0 + (long long)u * THREADS * VEC;
-            if (j < R.n) xor_into<VEC>(x[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+            x[u] = (R.coded_off >= 0 && j < end) ? load_words<VEC>(p.coded_in + R.coded_off + j)
+                                                 : zero_words<VEC>();
         }
-    }
+        for (int a = 0; a < p.na; ++a) {
+            const ccdc_ref E = sh_refs[a];
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        const long long j = j0 + (long long)u * THREADS * VEC;
-        if (j < R.n) store_words<VEC>(dst + j, x[u]);
+            for (int u = 0; u < UNROLL; ++u) {
+                const long long j = j0 + (long long)u * THREADS * VEC;
+                if (j < end) xor_into<VEC>(x[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const long long j = j0 + (long long)u * THREADS * VEC;
+            if (j < end) store_words<VEC>(dst + j, x[u]);
+        }
     }
 }
 
@@ -335,8 +342,13 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
         const long long tile = (long long)THREADS * VEC * UNROLL;
-        gp.tiles_per_row = (T.n_max + tile - 1) / tile;
-        const long long blocks = gp.nrows * gp.tiles_per_row;
+        // a block covers up to 16 tiles of a row, fewer while that would
+        // leave the grid short of 148 SMs x 16 blocks
+        long long tiles = 16;
+        while (tiles > 1 && gp.nrows * ((T.n_max + tile * tiles - 1) / (tile * tiles)) < 148 * 16) tiles /= 2;
+        gp.span_elems = tile * tiles;
+        gp.spans_per_row = (T.n_max + gp.span_elems - 1) / gp.span_elems;
+        const long long blocks = gp.nrows * gp.spans_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         k_gather<VEC, F32><<<(unsigned)blocks, THREADS, 0, st>>>(gp);
         return check_launch();
