@@ -6,16 +6,24 @@
 
 #include "ccdc.h"
 
-// launch shape shared by the planner (which sizes the split of the fused
-// decode from it) and the kernels
-#ifndef CCDC_THREADS_PER_BLOCK
-#define CCDC_THREADS_PER_BLOCK 256
+// Launch shapes (build-time options).  The fused decode+reduce keeps its loads
+// in registers; the gather kernel streams through a shared-memory pipeline.
+// The planner sizes the split of the fused decode from the decode tile.
+#ifndef CCDC_DECODE_THREADS
+#define CCDC_DECODE_THREADS 512     // threads per block
 #endif
-#ifndef CCDC_VECTORS_PER_THREAD
-#define CCDC_VECTORS_PER_THREAD 2
+#ifndef CCDC_DECODE_VECTORS
+#define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
-constexpr int CCDC_THREADS = CCDC_THREADS_PER_BLOCK;   // threads per block
-constexpr int CCDC_UNROLL = CCDC_VECTORS_PER_THREAD;   // vectors per thread per tile
+#ifndef CCDC_GATHER_THREADS
+#define CCDC_GATHER_THREADS 128
+#endif
+#ifndef CCDC_GATHER_VECTORS
+#define CCDC_GATHER_VECTORS 4       // vectors per thread per chunk
+#endif
+#ifndef CCDC_GATHER_STAGES
+#define CCDC_GATHER_STAGES 4        // chunks in flight per thread
+#endif
 
 // One operand of a gathered segment: element offset into the owning node's
 // buffer (segment offset included) and the number of leading elements of the

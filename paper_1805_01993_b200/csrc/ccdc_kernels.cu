@@ -17,8 +17,12 @@
 
 namespace {
 
-constexpr int THREADS = CCDC_THREADS;
-constexpr int UNROLL = CCDC_UNROLL;
+// launch shapes: D* = fused decode+reduce and the stepwise reduce, G* = gather
+constexpr int DTHREADS = CCDC_DECODE_THREADS;
+constexpr int DUNROLL = CCDC_DECODE_VECTORS;
+constexpr int GTHREADS = CCDC_GATHER_THREADS;
+constexpr int GUNROLL = CCDC_GATHER_VECTORS;
+constexpr int STAGES = CCDC_GATHER_STAGES;
 
 thread_local int g_last_cuda_error = 0;
 std::atomic<int> g_launches{0};
@@ -95,10 +99,50 @@ __device__ __forceinline__ Words<VEC> batch_sum(const uint32_t *src, long long o
     return acc;
 }
 
+// ------------------------------------------------- asynchronous load pipeline
+// Every streaming kernel keeps STAGES chunks of global loads in flight per
+// thread without holding them in registers: a thread copies its own VEC words
+// of a chunk global -> shared with cp.async (no register staging, the thread
+// runs on), commits one group per chunk, and STAGES-1 chunks later waits for
+// that group and reads its own words back.  A thread only ever reads slots it
+// filled itself, so the data path needs no block-wide barrier, and nothing
+// here can wait on another thread: there is no flag or mbarrier to hang on.
+
+template <int VEC>
+__device__ __forceinline__ void async_copy(uint32_t *smem, const uint32_t *gmem) {
+    const unsigned addr = (unsigned)__cvta_generic_to_shared(smem);
+    if (VEC == 4) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(addr), "l"(gmem) : "memory");
+    else if (VEC == 2) asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(addr), "l"(gmem) : "memory");
+    else asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(addr), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// this thread's slot for vector u of a stage
+template <int VEC>
+__device__ __forceinline__ uint32_t *slot_of(uint32_t *slots, int stage, int u) {
+    return slots + ((size_t)(stage * GUNROLL + u) * GTHREADS + threadIdx.x) * VEC;
+}
+
+template <int VEC>
+__device__ __forceinline__ Words<VEC> read_slot(const uint32_t *p) {
+    using V = typename WordVec<VEC>::type;
+    V v = *reinterpret_cast<const V *>(p);
+    Words<VEC> out;
+    memcpy(out.w, &v, sizeof(V));
+    return out;
+}
+
+__host__ __device__ constexpr size_t slots_bytes(int vec) { return (size_t)STAGES * GUNROLL * GTHREADS * vec * 4; }
+
 // ---------------------------------------------------------------- gather
 // dst row = [coded row XOR] XOR over operands of the batch sums of a segment.
 // Serves pre-combining (1 operand), encoding (r operands) and the stepwise
-// decode (coded row and r-1 operands).
+// decode (coded row and r-1 operands).  A batch sum adds the b files of a
+// batch in ascending order starting from the first file's value (the
+// pre-combined value of Section IV-B) and is zero where the segment does not
+// exist.
 struct GatherParams {
     const uint32_t *src[CCDC_MAX_K];
     uint32_t *dst[CCDC_MAX_K];
@@ -113,10 +157,18 @@ struct GatherParams {
     int b;
 };
 
+// position in a block's chunk sequence: for each tile of the span, the coded
+// row (operand -1, if any), then operand a = 0..na-1, file f = 0..b-1
+struct GatherCursor {
+    long long base;
+    int a, f;
+};
+
 template <int VEC, bool F32>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(GTHREADS)
 k_gather(const __grid_constant__ GatherParams p) {
-    constexpr long long TILE = (long long)THREADS * VEC * UNROLL;
+    constexpr long long TILE = (long long)GTHREADS * VEC * GUNROLL;
+    extern __shared__ __align__(16) uint32_t slots[];
     __shared__ ccdc_ref sh_refs[CCDC_MAX_K];
     const long long item = blockIdx.x;
     const long long row = item / p.spans_per_row;
@@ -130,29 +182,64 @@ k_gather(const __grid_constant__ GatherParams p) {
     __syncthreads();
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
+    const int a0 = R.coded_off >= 0 ? -1 : 0;
+    const long long tj = (long long)threadIdx.x * VEC;
 
-    for (long long base = begin; base < end; base += TILE) {
-        const long long j0 = base + (long long)threadIdx.x * VEC;
-        Words<VEC> x[UNROLL];
+    auto advance = [&](GatherCursor &c) {
+        if (c.a >= 0 && ++c.f < p.b) return;
+        c.f = 0;
+        if (++c.a >= p.na) { c.a = a0; c.base += TILE; }
+    };
+    // global address and validity of this thread's vector u of the chunk at c
+    auto locate = [&](const GatherCursor &c, int u, const uint32_t *&g) -> bool {
+        const long long j = c.base + tj + (long long)u * GTHREADS * VEC;
+        if (c.a < 0) { g = p.coded_in + R.coded_off + j; return j < end; }
+        const ccdc_ref E = sh_refs[c.a];
+        g = src + E.off + c.f * p.file_stride + j;
+        return j < end && j < E.vl;
+    };
+    auto issue = [&](const GatherCursor &c, int stage) {
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const long long j = j0 + (long long)u * THREADS * VEC;
-            x[u] = (R.coded_off >= 0 && j < end) ? load_words<VEC>(p.coded_in + R.coded_off + j)
-                                                 : zero_words<VEC>();
+        for (int u = 0; u < GUNROLL; ++u) {
+            const uint32_t *g;
+            if (locate(c, u, g)) async_copy<VEC>(slot_of<VEC>(slots, stage, u), g);
         }
-        for (int a = 0; a < p.na; ++a) {
-            const ccdc_ref E = sh_refs[a];
+    };
+
+    GatherCursor ic{begin, a0, 0}, cc{begin, a0, 0};
+    for (int i = 0; i < STAGES - 1; ++i) {
+        if (ic.base < end) { issue(ic, i); advance(ic); }
+        async_commit();
+    }
+    Words<VEC> x[GUNROLL], sum[GUNROLL];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                const long long j = j0 + (long long)u * THREADS * VEC;
-                if (j < end) xor_into<VEC>(x[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+    for (int u = 0; u < GUNROLL; ++u) x[u] = sum[u] = zero_words<VEC>();
+    int stage = 0;
+    while (cc.base < end) {
+        if (ic.base < end) { issue(ic, stage == 0 ? STAGES - 1 : stage - 1); advance(ic); }
+        async_commit();
+        async_wait<STAGES - 1>();
+        const bool last_file = cc.a < 0 || cc.f == p.b - 1;
+        const bool last_of_tile = last_file && cc.a == p.na - 1;
+#pragma unroll
+        for (int u = 0; u < GUNROLL; ++u) {
+            const uint32_t *g;
+            const bool ok = locate(cc, u, g);
+            const Words<VEC> v = ok ? read_slot<VEC>(slot_of<VEC>(slots, stage, u)) : zero_words<VEC>();
+            if (cc.a < 0) {
+                x[u] = v;
+            } else {
+                if (cc.f == 0) sum[u] = v; else add_into<VEC, F32>(sum[u], v);
+                if (last_file) xor_into<VEC>(x[u], sum[u]);
+            }
+            if (last_of_tile) {
+                const long long j = cc.base + tj + (long long)u * GTHREADS * VEC;
+                if (j < end) store_words<VEC>(dst + j, x[u]);
+                x[u] = zero_words<VEC>();
             }
         }
-#pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const long long j = j0 + (long long)u * THREADS * VEC;
-            if (j < end) store_words<VEC>(dst + j, x[u]);
-        }
+        advance(cc);
+        stage = stage + 1 == STAGES ? 0 : stage + 1;
     }
 }
 
@@ -178,9 +265,9 @@ struct DecodeParams {
 };
 
 template <int VEC, bool F32>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(DTHREADS)
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
-    constexpr long long TILE = (long long)THREADS * VEC * UNROLL;
+    constexpr long long TILE = (long long)DTHREADS * VEC * DUNROLL;
     extern __shared__ ccdc_ref sh_terms[];
 
     long long item = blockIdx.x;
@@ -201,60 +288,60 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
     const long long t_end = min(p.nterm, t_begin + p.terms_per_chunk);
     const ccdc_ref *table = p.terms + ((orow * p.r + i) * p.nterm) * p.TS;
 
-    Words<VEC> acc[UNROLL];
+    Words<VEC> acc[DUNROLL];
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) acc[u] = zero_words<VEC>();
+    for (int u = 0; u < DUNROLL; ++u) acc[u] = zero_words<VEC>();
 
     for (long long t0 = t_begin; t0 < t_end; t0 += p.stage_terms) {
         const int nt = (int)min((long long)p.stage_terms, t_end - t0);
         __syncthreads();
-        for (int x = threadIdx.x; x < nt * p.TS; x += THREADS) sh_terms[x] = table[t0 * p.TS + x];
+        for (int x = threadIdx.x; x < nt * p.TS; x += DTHREADS) sh_terms[x] = table[t0 * p.TS + x];
         __syncthreads();
         for (int t = 0; t < nt; ++t) {
             const ccdc_ref *e = sh_terms + t * p.TS;
             const long long coded_off = e[0].off;
-            Words<VEC> v[UNROLL];
+            Words<VEC> v[DUNROLL];
             if (coded_off < 0) {
                 const ccdc_ref E = e[1];
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const long long j = j0 + (long long)u * THREADS * VEC;
+                for (int u = 0; u < DUNROLL; ++u) {
+                    const long long j = j0 + (long long)u * DTHREADS * VEC;
                     v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
                 }
             } else {
 #pragma unroll
-                for (int u = 0; u < UNROLL; ++u) {
-                    const long long j = j0 + (long long)u * THREADS * VEC;
+                for (int u = 0; u < DUNROLL; ++u) {
+                    const long long j = j0 + (long long)u * DTHREADS * VEC;
                     v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
                 }
                 for (int c = 1; c <= r1; ++c) {
                     const ccdc_ref E = e[c];
 #pragma unroll
-                    for (int u = 0; u < UNROLL; ++u) {
-                        const long long j = j0 + (long long)u * THREADS * VEC;
+                    for (int u = 0; u < DUNROLL; ++u) {
+                        const long long j = j0 + (long long)u * DTHREADS * VEC;
                         if (j < seglen)
                             xor_into<VEC>(v[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
                     }
                 }
             }
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
+            for (int u = 0; u < DUNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
         }
     }
     uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) +
                     orow * p.len + (long long)i * p.s;
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-        const long long j = j0 + (long long)u * THREADS * VEC;
+    for (int u = 0; u < DUNROLL; ++u) {
+        const long long j = j0 + (long long)u * DTHREADS * VEC;
         if (j < seglen) store_words<VEC>(dst + j, acc[u]);
     }
 }
 
 // final pass of the split batch loop: out = ((ws[0] + ws[1]) + ...) in chunk order
 template <bool F32>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(DTHREADS)
 k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, long long n, int nchunk) {
-    const long long e = (long long)blockIdx.x * THREADS + threadIdx.x;
+    const long long e = (long long)blockIdx.x * DTHREADS + threadIdx.x;
     if (e >= n) return;
     uint32_t acc = ws[e];
     for (int c = 1; c < nchunk; ++c) acc = add_word<F32>(acc, ws[(long long)c * n + e]);
@@ -274,9 +361,9 @@ struct ReduceParams {
 };
 
 template <int VEC, bool F32>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(DTHREADS)
 k_reduce(const __grid_constant__ ReduceParams p) {
-    constexpr long long TILE = (long long)THREADS * VEC;
+    constexpr long long TILE = (long long)DTHREADS * VEC;
     const long long orow = blockIdx.x / p.tiles_per_row;
     const long long tile = blockIdx.x - orow * p.tiles_per_row;
     if (orow >= p.nout) return;
@@ -311,6 +398,15 @@ int check_launch() {
     return e == cudaSuccess ? CCDC_OK : cuda_fail(e);
 }
 
+// kernels that stage more than the default 48 KiB of dynamic shared memory
+// must opt in (a function attribute; nothing is allocated)
+template <typename Kernel>
+int allow_shared_memory(Kernel kernel, size_t bytes) {
+    if (bytes <= 32 * 1024) return CCDC_OK;         // static shared memory shares the 48 KiB default
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    return e == cudaSuccess ? CCDC_OK : cuda_fail(e);
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_ptr_array(const ccdc_plan_s &P, const void *const *a, bool (*nonempty)(const ccdc_plan_s &, int)) {
@@ -341,16 +437,19 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const long long tile = (long long)THREADS * VEC * UNROLL;
-        // a block covers up to 16 tiles of a row, fewer while that would
+        const long long tile = (long long)GTHREADS * VEC * GUNROLL;
+        // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 148 SMs x 16 blocks
-        long long tiles = 16;
+        long long tiles = 32;
         while (tiles > 1 && gp.nrows * ((T.n_max + tile * tiles - 1) / (tile * tiles)) < 148 * 16) tiles /= 2;
         gp.span_elems = tile * tiles;
         gp.spans_per_row = (T.n_max + gp.span_elems - 1) / gp.span_elems;
         const long long blocks = gp.nrows * gp.spans_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
-        k_gather<VEC, F32><<<(unsigned)blocks, THREADS, 0, st>>>(gp);
+        const size_t smem = slots_bytes(VEC);
+        int rc = allow_shared_memory(k_gather<VEC, F32>, smem);
+        if (rc != CCDC_OK) return rc;
+        k_gather<VEC, F32><<<(unsigned)blocks, GTHREADS, smem, st>>>(gp);
         return check_launch();
     });
 }
@@ -471,11 +570,11 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const long long tile = (long long)THREADS * VEC;
+        const long long tile = (long long)DTHREADS * VEC;
         rp.tiles_per_row = (P.len + tile - 1) / tile;
         const long long blocks = rp.nout * rp.tiles_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
-        k_reduce<VEC, F32><<<(unsigned)blocks, THREADS, 0, st>>>(rp);
+        k_reduce<VEC, F32><<<(unsigned)blocks, DTHREADS, 0, st>>>(rp);
         return check_launch();
     });
 }
@@ -510,19 +609,19 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
     dp.K = P.K; dp.r = P.r; dp.b = (int)P.b; dp.TS = P.term_stride; dp.nchunk = P.nchunk;
     const int stage_refs = 1024;                                    // 16 KiB of shared memory
     dp.stage_terms = (int)std::max(1LL, std::min<long long>(stage_refs / P.term_stride, P.terms_per_chunk));
-    const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const long long tile = (long long)THREADS * VEC * UNROLL;
+        const long long tile = (long long)DTHREADS * VEC * DUNROLL;
         dp.tiles_per_seg = (P.s + tile - 1) / tile;
         const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
-        k_decode_reduce<VEC, F32><<<(unsigned)blocks, THREADS, smem, st>>>(dp);
+        const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
+        k_decode_reduce<VEC, F32><<<(unsigned)blocks, DTHREADS, smem, st>>>(dp);
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
         const long long n = dp.nout * P.len;
-        k_sum_chunks<F32><<<(unsigned)((n + THREADS - 1) / THREADS), THREADS, 0, st>>>(dp.ws, dp.out, n, P.nchunk);
+        k_sum_chunks<F32><<<(unsigned)((n + DTHREADS - 1) / DTHREADS), DTHREADS, 0, st>>>(dp.ws, dp.out, n, P.nchunk);
         return check_launch();
     });
 }

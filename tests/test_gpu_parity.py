@@ -230,7 +230,7 @@ def sampled_full_size_check(ccdc, w, offsets_per_segment=48, seed=5):
     plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
     s = plan.segment_elems
     rng = np.random.default_rng(seed)
-    tile = 256 * 4 * 2
+    tile = 2048
     fixed = [0, 1, 3, s - 1, s - 4, min(tile - 1, s - 1), min(tile, s - 1), s // 2]
     offs = np.unique(np.concatenate([np.array(fixed), rng.integers(0, s, offsets_per_segment)]))
     m = len(offs)
