@@ -34,6 +34,26 @@ from paper_1805_01993_b200.inputs import CONFIGS, DEFAULT_SEED, values_numpy, va
 METRIC = "shuffle GB/s (combine+encode+decode+reduce)"
 UNIT = "GB/s"
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one k_decode_reduce
+# launch from the ncu capture summarised in profiles/k_decode_reduce_cfg4_B128000.md,
+# taken on the cfg4 structure with B = 128000; it grows in proportion to B.  Only
+# valid for the kernel sources it was measured on (hash below); otherwise null.
+NCU_TRAFFIC = {
+    "sources_sha256": "7faa876b7f3576e4c8b7d645ab3dc195f0432226f22e2a7756aa0fbbecba7f1c",
+    "workload": "cfg4", "value_elems": 128000, "decode_kernel_bytes": 3.537435e9 + 28.169984e6,
+}
+
+
+def measured_traffic(w):
+    import hashlib
+
+    h = hashlib.sha256()
+    for f in ("ccdc_kernels.cu", "ccdc_internal.h"):
+        h.update((ROOT / "paper_1805_01993_b200" / "csrc" / f).read_bytes())
+    if h.hexdigest() != NCU_TRAFFIC["sources_sha256"] or not w.name.startswith(NCU_TRAFFIC["workload"]):
+        return None
+    return NCU_TRAFFIC["decode_kernel_bytes"] * w.B / NCU_TRAFFIC["value_elems"]
+
 
 # ---------------------------------------------------------------- byte counts
 def algorithmic_bytes(K, r, N, Q, B, J=1, rounds=None):
@@ -280,10 +300,7 @@ def run_ours(args, w):
         peak, peak_kind = 6650.0, "fallback"
     achieved = by["decode_kernel"] / (dec_ms * 1e-3) / 1e9
     enc_achieved = by["encode_kernel"] / (enc_ms * 1e-3) / 1e9
-    traffic_file = ROOT / "profiles" / "traffic.json"
-    traffic = None
-    if traffic_file.exists():
-        traffic = json.loads(traffic_file.read_text()).get("decode_kernel_bytes_per_launch")
+    traffic = measured_traffic(w)
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
