@@ -132,6 +132,29 @@ size_t ccdc_workspace_bytes(const ccdc_plan_t *plan);         /* ccdc_shuffle sc
 /* ------------------------------------------------------------------ steps
  * part, packets, decoded: device pointer arrays (see above). */
 
+/* Map phase (Section III, "Map phase") of the linear-regression workload: for
+ * every file n stored at node k, the Q intermediate values v_{q,n} are the Q
+ * contiguous slices of the partial gradient
+ *     g_n = X_n^T (X_n w - y_n),   X_n [rows][d] bf16 row-major, d = Q*B,
+ *     y_n [rows] fp32, w [d] bf16,
+ * computed with bf16 tensor-core products accumulated in fp32 (the fp32
+ * residual enters the second product as the sum of three bf16 terms, so no
+ * precision is lost to the operand format) and written as fp32 into part[k] in
+ * the partition layout.  Every node maps its own copy of a file; replicas are
+ * bit-identical because the same deterministic kernels, with one fixed
+ * summation order, run for each.
+ *   files_x[k]: node k's files, [local batch][file in batch][rows][d] bf16
+ *   files_y[k]: [local batch][file in batch][rows] fp32
+ *   w: device pointer, [d] bf16;  workspace: ccdc_map_workspace_bytes(plan, rows)
+ *   (the residuals; fully written before read).
+ * F32 plans only (CCDC_ESTATE otherwise).  CCDC_ESIZE unless rows is a multiple
+ * of 16 in 16..4096 and d a multiple of 512 up to 65536.  Asynchronous on
+ * `stream`; launches two kernels per wave of files (a wave is sized to stay in
+ * L2 between the two products). */
+size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows);
+int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
+             long long rows, void *const *part, void *workspace, void *stream);
+
 /* Pre-combining (Section IV-B): packets[k][local batch][t] = concatenation over
  * q in S_t of  sum_{n in batch} v_{q,n}, files added in ascending order
  * starting from the first file's value. */

@@ -48,6 +48,8 @@ SIGNATURES = {
     "ccdc_coded_bytes": (_SZ, [_P]),
     "ccdc_out_bytes": (_SZ, [_P]),
     "ccdc_workspace_bytes": (_SZ, [_P]),
+    "ccdc_map_workspace_bytes": (_SZ, [_P, _LL]),
+    "ccdc_map": (_I, [_P, _PP, _PP, _P, _LL, _PP, _P, _P]),
     "ccdc_combine": (_I, [_P, _PP, _PP, _P]),
     "ccdc_encode": (_I, [_P, _PP, _P, _P]),
     "ccdc_decode": (_I, [_P, _PP, _P, _PP, _P]),
@@ -247,6 +249,14 @@ class Plan:
         return sampled
 
     # ---- steps ------------------------------------------------------------
+    def map_workspace_bytes(self, rows):
+        return lib().ccdc_map_workspace_bytes(self._h, rows)
+
+    def map(self, files_x, files_y, w, rows, part, workspace, stream=None):
+        """``files_x`` / ``files_y``: per node, bf16 ``[files][rows][Q*B]`` and fp32 ``[files][rows]``."""
+        _check(lib().ccdc_map(self._h, _ptr_array(files_x), _ptr_array(files_y), w.data_ptr(), rows,
+                              _ptr_array(part), workspace.data_ptr(), _stream_handle(stream)), "ccdc_map")
+
     def combine(self, part, packets, stream=None):
         _check(lib().ccdc_combine(self._h, _ptr_array(part), _ptr_array(packets), _stream_handle(stream)),
                "ccdc_combine")

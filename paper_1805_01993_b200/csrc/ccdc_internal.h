@@ -101,3 +101,5 @@ struct ccdc_plan_s {
 
 // implemented in ccdc_kernels.cu
 void ccdc_internal_release_device(ccdc_plan_s *plan);
+int ccdc_internal_cuda_fail(int cuda_error);    // records the error for ccdc_last_cuda_error; returns CCDC_ECUDA
+void ccdc_internal_count_launch();              // one more kernel launched by the library

@@ -465,6 +465,9 @@ int ensure_device(ccdc_plan_s *plan) {
 
 }  // namespace
 
+int ccdc_internal_cuda_fail(int cuda_error) { return cuda_fail((cudaError_t)cuda_error); }
+void ccdc_internal_count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
 void ccdc_internal_release_device(ccdc_plan_s *plan) {
     if (plan->d_blob) {
         int cur = -1;

@@ -1,0 +1,133 @@
+"""Parity of the tensor-core Map (partial gradients of linear regression) and of
+the whole job Map -> shuffle -> reduce with the CPU oracle.
+
+The oracle evaluates g = X^T (X w - y) in binary64 on the same bf16-representable
+X and w and rounds once to fp32.  The CUDA Map accumulates bf16 products in fp32,
+so its values agree to fp32 accumulation error, not bit for bit; what must hold
+exactly is that the r replicas of a file's values are bit-identical (XOR decoding
+depends on it).  Tolerances:
+  Map value j:      |gpu - oracle| <= 1e-5 * sum_i |X_ij| |u_i|
+  Reduce output:    |gpu - oracle| <= 1e-5 * sum_n |v_{q,n}|   (the evaluation's rule)
+"""
+import numpy as np
+import pytest
+
+from oracle.ccdc_oracle import Oracle, map_linear_regression
+from paper_1805_01993_b200.inputs import CONFIGS, bf16_bits, regression_files
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def ccdc():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_1805_01993_b200 import build, ccdc as mod
+
+    build.build_library()
+    mod.lib()
+    return mod
+
+
+def to_bf16_cuda(a):
+    return torch.from_numpy(bf16_bits(a).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def run_job(ccdc, K, r, N, Q, B, rows, seed):
+    d = Q * B
+    X, y, w = regression_files(N, rows, d, seed=seed)
+    plan = ccdc.Plan(K, r, N, Q, B, "float32")
+    # ---- oracle: Map in binary64, then the scheme
+    v = np.stack([map_linear_regression(X[n], w, y[n], Q) for n in range(N)])
+    o = Oracle(K, r, N, Q, B, "float32")
+    ref_out = o.run(v)
+    # ---- CUDA: every node maps its own copy of its files
+    files_x, files_y = [], []
+    for k in range(K):
+        idx = plan.node_files(k)
+        files_x.append(to_bf16_cuda(X[idx]).contiguous())
+        files_y.append(torch.from_numpy(y[idx]).cuda().contiguous())
+    wd = to_bf16_cuda(w)
+    part = plan.alloc_partitions()
+    for p in part:
+        p.fill_(float("nan"))
+    ws = torch.empty(plan.map_workspace_bytes(rows) // 4, dtype=torch.float32, device="cuda")
+    before = ccdc.num_kernel_launches()
+    plan.map(files_x, files_y, wd, rows, part, ws)
+    torch.cuda.synchronize()
+    assert ccdc.num_kernel_launches() - before >= 2
+    # Map values against the oracle, and replicas against each other
+    Xd = X.astype(np.float64)
+    u = np.einsum("nij,j->ni", Xd, w.astype(np.float64)) - y.astype(np.float64)
+    scale = np.einsum("nij,ni->nj", np.abs(Xd), np.abs(u))            # sum_i |X_ij||u_i|
+    first = {}
+    worst = 0.0
+    for k in range(K):
+        got = part[k].cpu().numpy().reshape(-1, d)
+        for i, n in enumerate(plan.node_files(k)):
+            err = np.abs(got[i].astype(np.float64) - v[n].reshape(-1))
+            assert np.all(err <= 1e-5 * scale[n]), (k, n, float((err / scale[n]).max()))
+            worst = max(worst, float((err / scale[n]).max()))
+            if n in first:
+                assert np.array_equal(first[n].view(np.uint32), got[i].view(np.uint32)), \
+                    f"replicas of file {n} differ"
+            else:
+                first[n] = got[i].copy()
+    assert len(first) == N
+    # ---- shuffle + reduce on the mapped partitions
+    coded = plan.alloc(plan.coded_bytes)
+    out = plan.alloc(plan.out_bytes)
+    wsp = plan.alloc(plan.workspace_bytes)
+    plan.shuffle(part, coded, out, wsp)
+    torch.cuda.synchronize()
+    got_out = out.cpu().numpy().reshape(Q, B)
+    _, a64 = o.direct()
+    err = np.abs(got_out.astype(np.float64) - ref_out.astype(np.float64))
+    assert np.all(err <= 1e-5 * a64), float((err / a64).max())
+    # the full gradient: sum over all files, against binary64
+    full = np.einsum("nij,ni->j", Xd, u).reshape(Q, B)
+    assert np.all(np.abs(got_out - full) <= 1e-5 * a64)
+    # exact consistency on the device side: the shuffle of the GPU's own Map values
+    # must reproduce their fixed-order sum (decode loses nothing)
+    mine = np.stack([first[n].reshape(Q, B) for n in range(N)])
+    o2 = Oracle(K, r, N, Q, B, "float32")
+    ref2 = o2.run(mine)
+    s, sp = plan.segment_elems, plan.coded_row_elems
+    assert np.array_equal(coded.cpu().numpy().view(np.uint32).reshape(-1, sp)[:, :s], o2.coded().reshape(-1, s))
+    _, a2 = o2.direct()
+    assert np.all(np.abs(got_out.astype(np.float64) - ref2) <= 1e-5 * a2)
+    return worst
+
+
+def test_map_small(ccdc):
+    worst = run_job(ccdc, 4, 2, 12, 4, 128, rows=32, seed=7)
+    assert worst < 1e-5
+
+
+def test_map_wide_files(ccdc):
+    # d = 2048 columns, 48 rows, r = K-1
+    run_job(ccdc, 4, 3, 8, 4, 512, rows=48, seed=8)
+
+
+def test_cfg5_full_job(ccdc):
+    w = CONFIGS["cfg5"]
+    worst = run_job(ccdc, w.K, w.r, w.N, w.Q, w.B, rows=w.map_rows, seed=9)
+    assert worst < 1e-5
+
+
+def test_map_refuses_bad_shapes(ccdc):
+    plan = ccdc.Plan(4, 2, 12, 4, 128, "float32")
+    z = torch.zeros(16, device="cuda")
+    with pytest.raises(ccdc.CcdcError) as e:
+        plan.map([z] * 4, [z] * 4, z, 24, [z] * 4, z)          # rows not a multiple of 16
+    assert e.value.status == ccdc.ESIZE
+    iplan = ccdc.Plan(4, 2, 12, 4, 128, "int32")
+    with pytest.raises(ccdc.CcdcError) as e:
+        iplan.map([z] * 4, [z] * 4, z, 32, [z] * 4, z)
+    assert e.value.status == ccdc.ESTATE
+    odd = ccdc.Plan(4, 2, 12, 4, 100, "float32")               # d = 400 is not a multiple of 512
+    with pytest.raises(ccdc.CcdcError) as e:
+        odd.map([z] * 4, [z] * 4, z, 32, [z] * 4, z)
+    assert e.value.status == ccdc.ESIZE
