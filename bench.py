@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # taken on the cfg4 structure with B = 128000; it grows in proportion to B.  Only
 # valid for the kernel sources it was measured on (hash below); otherwise null.
 NCU_TRAFFIC = {
-    "sources_sha256": "7faa876b7f3576e4c8b7d645ab3dc195f0432226f22e2a7756aa0fbbecba7f1c",
+    "sources_sha256": "b4edafd69a04024433cf3d7b0fa623f7464dd7ae9b6c85ef7e18c38ee678dbaf",
     "workload": "cfg4", "value_elems": 128000, "decode_kernel_bytes": 3.537435e9 + 28.169984e6,
 }
 
@@ -211,41 +211,74 @@ def run_ours(args, w):
     plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
     plan.upload()
     part = plan.alloc_partitions(dev)
-    # every rank is an independent job of the same shape: its own seed
-    plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=DEFAULT_SEED + rank,
-                                                      std=w.std))
     coded = plan.alloc(plan.coded_bytes, dev)
     out = plan.alloc(plan.out_bytes, dev)
     ws = plan.alloc(plan.workspace_bytes, dev)
     by = algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B)
     stream = torch.cuda.current_stream()
+    stages = []
+    map_bytes = 0
+    if w.map_rows:
+        # linear-regression workload: the partitions are produced by the Map, which is
+        # part of the step (job time = Map + shuffle); files drawn on the device
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(DEFAULT_SEED + rank)
+        d = w.Q * w.B
+        canon = torch.randn((w.N, w.map_rows, d), generator=gen, device=dev).to(torch.bfloat16)
+        ycan = torch.randn((w.N, w.map_rows), generator=gen, device=dev)
+        files_x = [canon[plan.node_files(k)].contiguous() for k in range(w.K)]
+        files_y = [ycan[plan.node_files(k)].contiguous() for k in range(w.K)]
+        del canon, ycan
+        wvec = torch.randn(d, generator=gen, device=dev).to(torch.bfloat16)
+        map_ws = torch.empty(plan.map_workspace_bytes(w.map_rows) // 4, dtype=torch.float32, device=dev)
+        map_bytes = sum(t.numel() * 2 for t in files_x) + sum(plan.partition_bytes(k) for k in range(w.K))
+        stages.append(("k_map_residual+k_map_gradient",
+                       lambda: plan.map(files_x, files_y, wvec, w.map_rows, part, map_ws)))
+    else:
+        # every rank is an independent job of the same shape: its own seed
+        plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=DEFAULT_SEED + rank,
+                                                          std=w.std))
+    stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
+    stages.append(("k_decode_reduce", lambda: plan.decode_reduce(part, coded, out, ws)))
+    stage_bytes = {"k_map_residual+k_map_gradient": map_bytes, "k_gather(encode)": by["encode_kernel"],
+                   "k_decode_reduce": by["decode_kernel"]}
+    input_bytes = sum(plan.partition_bytes(k) for k in range(w.K)) + map_bytes
+    # inputs that fit in L2 (126 MB) would be served from it on every repeat: flush between steps
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if input_bytes < (1 << 30) else None
+
+    def one_step(events=None):
+        if flush is not None:
+            flush.zero_()
+        for i, (_, fn) in enumerate(stages):
+            if events is not None:
+                events[i].record(stream)
+            fn()
+        if events is not None:
+            events[len(stages)].record(stream)
 
     for _ in range(args.warmup):
-        plan.shuffle(part, coded, out, ws)
+        one_step()
     barrier()
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(stages) + 1)] for _ in range(args.steps)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = ccdc.num_kernel_launches()
     barrier()
     start.record(stream)
     for i in range(args.steps):
-        ev[i][0].record(stream)
-        plan.encode_fused(part, coded)
-        ev[i][1].record(stream)
-        plan.decode_reduce(part, coded, out, ws)
-        ev[i][2].record(stream)
+        one_step(ev[i])
     end.record(stream)
     barrier()
     launches = ccdc.num_kernel_launches() - launches0
     clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = start.elapsed_time(end)
-    enc_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
-    dec_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    # with a flush between steps the bracket would include it: sum the steps instead
+    elapsed_ms = start.elapsed_time(end) if flush is None else sum(e[0].elapsed_time(e[-1]) for e in ev)
+    stage_ms = {name: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
+    enc_ms, dec_ms = stage_ms["k_gather(encode)"], stage_ms["k_decode_reduce"]
     t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -257,6 +290,8 @@ def run_ours(args, w):
     try:
         if args.skip_e2e:
             raise RuntimeError("--skip-e2e")
+        if w.map_rows:
+            raise RuntimeError("host-buffer leg is defined for the shuffle-only workloads")
         import psutil
 
         need = sum(plan.partition_bytes(k) for k in range(w.K)) + plan.out_bytes
@@ -298,9 +333,12 @@ def run_ours(args, w):
         peak, peak_kind = json.loads(peaks_file.read_text())["hbm_gbs"], "measured"
     else:
         peak, peak_kind = 6650.0, "fallback"
-    achieved = by["decode_kernel"] / (dec_ms * 1e-3) / 1e9
-    enc_achieved = by["encode_kernel"] / (enc_ms * 1e-3) / 1e9
-    traffic = measured_traffic(w)
+    top = max(stage_ms, key=stage_ms.get)                 # the dominant kernel of the step
+    achieved = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
+    others = {n: {"achieved": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9,
+                  "frac": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / peak, "ms_per_launch": stage_ms[n]}
+              for n in stage_ms if n != top}
+    traffic = measured_traffic(w) if top == "k_decode_reduce" else None
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -316,15 +354,15 @@ def run_ours(args, w):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
-                   "l2": f"inputs ({sum(plan.partition_bytes(k) for k in range(w.K)) / 1e9:.1f} GB) larger than L2, no flush", "jobs_per_gpu": 1,
+                   "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
+                          f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written between steps, steps timed one by one"),
+                   "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": 1,
                    "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
-                   "algorithmic_bytes_per_step": by["total"],
-                   "hbm_frac_whole_step": by["total"] / (ms_per_step * 1e-3) / 1e9 / peak},
-        "roofline": {"bound": "hbm", "kernel": "k_decode_reduce", "achieved": achieved, "peak": peak,
+                   "algorithmic_bytes_per_step": by["total"] + map_bytes,
+                   "hbm_frac_whole_step": (by["total"] + map_bytes) / (ms_per_step * 1e-3) / 1e9 / peak},
+        "roofline": {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
-                     "ms_per_launch": dec_ms,
-                     "other_kernels": {"k_gather(encode)": {"achieved": enc_achieved, "frac": enc_achieved / peak,
-                                                            "ms_per_launch": enc_ms}}},
+                     "ms_per_launch": stage_ms[top], "other_kernels": others},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
     }
     print(json.dumps(line))

@@ -149,8 +149,7 @@ size_t ccdc_workspace_bytes(const ccdc_plan_t *plan);         /* ccdc_shuffle sc
  *   (the residuals; fully written before read).
  * F32 plans only (CCDC_ESTATE otherwise).  CCDC_ESIZE unless rows is a multiple
  * of 16 in 16..4096 and d a multiple of 512 up to 65536.  Asynchronous on
- * `stream`; launches two kernels per wave of files (a wave is sized to stay in
- * L2 between the two products). */
+ * `stream`; two kernel launches (one per product). */
 size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows);
 int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
              long long rows, void *const *part, void *workspace, void *stream);

@@ -10,7 +10,6 @@
 //   pass 2  g = X^T u          A = u split into three bf16 terms (rows 0..2),
 //                              B = 16 rows x 8 columns of X, packed from four
 //                              row vectors with byte permutes
-// Files are processed in waves small enough for pass 2 to find X_n in L2.
 // Every node maps its own copy of a file with the same code and the same fixed
 // summation order, so the replicas are bit-identical (no atomics anywhere).
 #include <cuda_bf16.h>
@@ -24,6 +23,14 @@
 
 namespace {
 
+// Files can be mapped in waves whose X stays in L2 between the two passes
+// (CCDC_MAP_WAVE_MB > 0).  Measured on B200 that loses: grids of a wave are too
+// small to saturate HBM (1.48 ms at 96 MB per wave against 0.92 ms for one wave
+// over all 336 files of the K = 8 workload, where each pass streams X at the
+// HBM rate).  0 = one wave.
+#ifndef CCDC_MAP_WAVE_MB
+#define CCDC_MAP_WAVE_MB 0
+#endif
 constexpr int MAP_THREADS = 256;                 // pass 1: 8 warps share 16 rows
 constexpr int MAP_WARPS = MAP_THREADS / 32;
 constexpr int GRAD_THREADS = 128;                // pass 2: 4 warps x 64 columns
@@ -243,9 +250,9 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
     mp.rows = rows; mp.d = d; mp.K = P.K;
     const long long njobs = mp.first_job[P.K];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // files per wave: pass 2 should still find the wave's X in L2 (126 MB)
     const long long file_bytes = rows * d * 2;
-    const long long wave = std::max(1LL, (96LL << 20) / file_bytes);
+    const long long wave = CCDC_MAP_WAVE_MB > 0 ? std::max(1LL, ((long long)CCDC_MAP_WAVE_MB << 20) / file_bytes)
+                                                : std::max(1LL, njobs);
     const size_t smem1 = (size_t)d * 2, smem2 = (size_t)rows * 6;
     if (smem1 > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(k_map_residual, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
