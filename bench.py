@@ -81,6 +81,28 @@ def algorithmic_bytes(K, r, N, Q, B, J=1, rounds=None):
     }
 
 
+# ---------------------------------------------------------------- multi-rank
+def rank_seed(rank: int) -> int:
+    """Every rank runs an independent job of the same shape: its own input seed."""
+    return DEFAULT_SEED + rank
+
+
+def max_over_ranks(ms: float, world: int, device):
+    """Slowest rank's time (the job is done when the last rank is)."""
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def whole_job_value(world: int, bytes_per_rank: int, ms_per_step: float) -> float:
+    """GB/s over all ranks: every rank moved bytes_per_rank in ms_per_step."""
+    return world * bytes_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 # ---------------------------------------------------------------- clocks
 class ClockSampler:
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -222,7 +244,7 @@ def run_ours(args, w):
         # linear-regression workload: the partitions are produced by the Map, which is
         # part of the step (job time = Map + shuffle); files drawn on the device
         gen = torch.Generator(device=dev)
-        gen.manual_seed(DEFAULT_SEED + rank)
+        gen.manual_seed(rank_seed(rank))
         d = w.Q * w.B
         canon = torch.randn((w.N, w.map_rows, d), generator=gen, device=dev).to(torch.bfloat16)
         ycan = torch.randn((w.N, w.map_rows), generator=gen, device=dev)
@@ -236,7 +258,7 @@ def run_ours(args, w):
                        lambda: plan.map(files_x, files_y, wvec, w.map_rows, part, map_ws)))
     else:
         # every rank is an independent job of the same shape: its own seed
-        plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=DEFAULT_SEED + rank,
+        plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=rank_seed(rank),
                                                           std=w.std))
     stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
     stages.append(("k_decode_reduce", lambda: plan.decode_reduce(part, coded, out, ws)))
@@ -279,11 +301,8 @@ def run_ours(args, w):
     elapsed_ms = start.elapsed_time(end) if flush is None else sum(e[0].elapsed_time(e[-1]) for e in ev)
     stage_ms = {name: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
     enc_ms, dec_ms = stage_ms["k_gather(encode)"], stage_ms["k_decode_reduce"]
-    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_per_step = t.item() / args.steps
-    value = world * by["iv_read"] / (ms_per_step * 1e-3) / 1e9
+    ms_per_step = max_over_ranks(elapsed_ms, world, dev) / args.steps
+    value = whole_job_value(world, by["iv_read"], ms_per_step)
 
     # ---- end to end through the host-buffer entry point ------------------
     e2e = None
@@ -309,12 +328,10 @@ def run_ours(args, w):
                 plan.shuffle_host(host_part, host_out, part, coded, out, ws)
             e2.record(stream)
             barrier()
-            t2 = torch.tensor([s2.elapsed_time(e2)], dtype=torch.float64, device=dev)
-            if world > 1:
-                dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-            e2e = {"value": world * by["iv_read"] / (t2.item() / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+            e2e_ms = max_over_ranks(s2.elapsed_time(e2), world, dev) / e2e_steps
+            e2e = {"value": whole_job_value(world, by["iv_read"], e2e_ms), "unit": UNIT,
                    "h2d_bytes_per_step": need - plan.out_bytes, "d2h_bytes_per_step": plan.out_bytes,
-                   "steps": e2e_steps, "ms_per_step": t2.item() / e2e_steps}
+                   "steps": e2e_steps, "ms_per_step": e2e_ms}
             assert torch.equal(host_out, out.cpu())
             del host_part
         else:

@@ -12,6 +12,9 @@
 #ifndef CCDC_DECODE_THREADS
 #define CCDC_DECODE_THREADS 512     // threads per block
 #endif
+#ifndef CCDC_DECODE_THREADS_SHORT
+#define CCDC_DECODE_THREADS_SHORT 1024  // used instead when one such block covers a whole segment
+#endif
 #ifndef CCDC_DECODE_VECTORS
 #define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
@@ -68,6 +71,7 @@ struct ccdc_plan_s {
     long long nbatch = 0, nround = 0, nterm = 0;   // nterm = batches per job
     int vec = 1;              // widest vector (words) dividing s and len: 4, 2 or 1
     int term_stride = 0;      // refs per term of the fused decode: 1 + max(r-1, 1)
+    int decode_threads = CCDC_DECODE_THREADS;   // block size of the fused decode
     int nchunk = 1;           // split of the batch loop in the fused decode
     long long terms_per_chunk = 0;
 

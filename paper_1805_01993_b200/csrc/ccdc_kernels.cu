@@ -264,10 +264,10 @@ struct DecodeParams {
     int stage_terms;        // terms staged in shared memory at a time
 };
 
-template <int VEC, bool F32>
-__global__ void __launch_bounds__(DTHREADS)
+template <int VEC, bool F32, int NT>
+__global__ void __launch_bounds__(NT)
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
-    constexpr long long TILE = (long long)DTHREADS * VEC * DUNROLL;
+    constexpr long long TILE = (long long)NT * VEC * DUNROLL;
     extern __shared__ ccdc_ref sh_terms[];
 
     long long item = blockIdx.x;
@@ -295,7 +295,7 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
     for (long long t0 = t_begin; t0 < t_end; t0 += p.stage_terms) {
         const int nt = (int)min((long long)p.stage_terms, t_end - t0);
         __syncthreads();
-        for (int x = threadIdx.x; x < nt * p.TS; x += DTHREADS) sh_terms[x] = table[t0 * p.TS + x];
+        for (int x = threadIdx.x; x < nt * p.TS; x += NT) sh_terms[x] = table[t0 * p.TS + x];
         __syncthreads();
         for (int t = 0; t < nt; ++t) {
             const ccdc_ref *e = sh_terms + t * p.TS;
@@ -305,20 +305,20 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                 const ccdc_ref E = e[1];
 #pragma unroll
                 for (int u = 0; u < DUNROLL; ++u) {
-                    const long long j = j0 + (long long)u * DTHREADS * VEC;
+                    const long long j = j0 + (long long)u * NT * VEC;
                     v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
                 }
             } else {
 #pragma unroll
                 for (int u = 0; u < DUNROLL; ++u) {
-                    const long long j = j0 + (long long)u * DTHREADS * VEC;
+                    const long long j = j0 + (long long)u * NT * VEC;
                     v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
                 }
                 for (int c = 1; c <= r1; ++c) {
                     const ccdc_ref E = e[c];
 #pragma unroll
                     for (int u = 0; u < DUNROLL; ++u) {
-                        const long long j = j0 + (long long)u * DTHREADS * VEC;
+                        const long long j = j0 + (long long)u * NT * VEC;
                         if (j < seglen)
                             xor_into<VEC>(v[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
                     }
@@ -332,7 +332,7 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                     orow * p.len + (long long)i * p.s;
 #pragma unroll
     for (int u = 0; u < DUNROLL; ++u) {
-        const long long j = j0 + (long long)u * DTHREADS * VEC;
+        const long long j = j0 + (long long)u * NT * VEC;
         if (j < seglen) store_words<VEC>(dst + j, acc[u]);
     }
 }
@@ -615,12 +615,15 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const long long tile = (long long)DTHREADS * VEC * DUNROLL;
+        const long long tile = (long long)P.decode_threads * VEC * DUNROLL;
         dp.tiles_per_seg = (P.s + tile - 1) / tile;
         const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
-        k_decode_reduce<VEC, F32><<<(unsigned)blocks, DTHREADS, smem, st>>>(dp);
+        if (P.decode_threads == CCDC_DECODE_THREADS_SHORT)
+            k_decode_reduce<VEC, F32, CCDC_DECODE_THREADS_SHORT><<<(unsigned)blocks, CCDC_DECODE_THREADS_SHORT, smem, st>>>(dp);
+        else
+            k_decode_reduce<VEC, F32, DTHREADS><<<(unsigned)blocks, DTHREADS, smem, st>>>(dp);
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
         const long long n = dp.nout * P.len;

@@ -236,7 +236,11 @@ int finish(ccdc_plan_s &P) {
     // fill the GPU (148 SMs x 8 resident blocks) while a block still walks a
     // fair number of batches
     {
-        const long long tile = (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS;
+        // short segments: one large block per segment beats two smaller ones (measured on K=16, r=4)
+        if (P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
+            P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS)
+            P.decode_threads = CCDC_DECODE_THREADS_SHORT;
+        const long long tile = (long long)P.decode_threads * P.vec * CCDC_DECODE_VECTORS;
         const long long tiles_per_seg = (P.s + tile - 1) / tile;
         const long long base = nout * r * tiles_per_seg;
         long long want = (148LL * 8 + base - 1) / base;
