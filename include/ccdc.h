@@ -146,13 +146,24 @@ size_t ccdc_workspace_bytes(const ccdc_plan_t *plan);         /* ccdc_shuffle sc
  *   files_x[k]: node k's files, [local batch][file in batch][rows][d] bf16
  *   files_y[k]: [local batch][file in batch][rows] fp32
  *   w: device pointer, [d] bf16;  workspace: ccdc_map_workspace_bytes(plan, rows)
- *   (the residuals; fully written before read).
+ *   (residuals plus a few control words; the call resets what it needs).
  * F32 plans only (CCDC_ESTATE otherwise).  CCDC_ESIZE unless rows is a multiple
  * of 16 in 16..4096 and d a multiple of 512 up to 65536.  Asynchronous on
- * `stream`; two kernel launches (one per product). */
+ * `stream`: one memset and ONE kernel launch.  Inside it, work items are handed
+ * out in order by an atomic ticket (per file its first-product blocks, then the
+ * second-product blocks of the previous file) so that the second product finds
+ * the file in L2; a second-product block polls a per-file counter until the
+ * file's residuals are complete.  The blocks it waits for hold smaller tickets,
+ * are therefore already running and wait on nothing, so the poll always ends;
+ * it is bounded anyway, and ccdc_map_status reports if a bound was ever hit.
+ *
+ * ccdc_map_status: call after the stream has been synchronised; copies one word
+ * back (synchronous) and returns CCDC_OK, or CCDC_ESTATE if a wait ran out (the
+ * Map results of that call are then not valid). */
 size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows);
 int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
              long long rows, void *const *part, void *workspace, void *stream);
+int ccdc_map_status(const ccdc_plan_t *plan, long long rows, const void *workspace);
 
 /* Pre-combining (Section IV-B): packets[k][local batch][t] = concatenation over
  * q in S_t of  sum_{n in batch} v_{q,n}, files added in ascending order

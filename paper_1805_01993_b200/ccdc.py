@@ -50,6 +50,7 @@ SIGNATURES = {
     "ccdc_workspace_bytes": (_SZ, [_P]),
     "ccdc_map_workspace_bytes": (_SZ, [_P, _LL]),
     "ccdc_map": (_I, [_P, _PP, _PP, _P, _LL, _PP, _P, _P]),
+    "ccdc_map_status": (_I, [_P, _LL, _P]),
     "ccdc_combine": (_I, [_P, _PP, _PP, _P]),
     "ccdc_encode": (_I, [_P, _PP, _P, _P]),
     "ccdc_decode": (_I, [_P, _PP, _P, _PP, _P]),
@@ -251,6 +252,10 @@ class Plan:
     # ---- steps ------------------------------------------------------------
     def map_workspace_bytes(self, rows):
         return lib().ccdc_map_workspace_bytes(self._h, rows)
+
+    def map_status(self, rows, workspace):
+        """after a synchronise: raises if a wait inside the Map kernel ran out."""
+        _check(lib().ccdc_map_status(self._h, rows, workspace.data_ptr()), "ccdc_map_status")
 
     def map(self, files_x, files_y, w, rows, part, workspace, stream=None):
         """``files_x`` / ``files_y``: per node, bf16 ``[files][rows][Q*B]`` and fp32 ``[files][rows]``."""

@@ -3,15 +3,15 @@
 // values are the Q contiguous slices of the partial gradient
 //     g_n = X_n^T (X_n w - y_n),        X_n [rows][d] bf16, d = Q*B.
 // Both products run on the tensor cores (mma.sync m16n8k16, bf16 operands, fp32
-// accumulators).  The shape is matrix-vector, so the kernels are bound by the
-// read of X_n; they are laid out so that every 16-byte load is coalesced and X_n
-// never passes through shared memory:
+// accumulators).  The shape is matrix-vector, so the work is bound by the read
+// of X_n; every 16-byte load is coalesced and X_n never passes through shared
+// memory:
 //   pass 1  u = X w - y        A = 16 rows of X (k = columns), B = w in column 0
 //   pass 2  g = X^T u          A = u split into three bf16 terms (rows 0..2),
 //                              B = 16 rows x 8 columns of X, packed from four
 //                              row vectors with byte permutes
 // Every node maps its own copy of a file with the same code and the same fixed
-// summation order, so the replicas are bit-identical (no atomics anywhere).
+// summation order, so the replicas are bit-identical (no floating-point atomics).
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -23,19 +23,25 @@
 
 namespace {
 
-// Files can be mapped in waves whose X stays in L2 between the two passes
-// (CCDC_MAP_WAVE_MB > 0).  Measured on B200 that loses: grids of a wave are too
-// small to saturate HBM (1.48 ms at 96 MB per wave against 0.92 ms for one wave
-// over all 336 files of the K = 8 workload, where each pass streams X at the
-// HBM rate).  0 = one wave.
-#ifndef CCDC_MAP_WAVE_MB
-#define CCDC_MAP_WAVE_MB 0
+#ifndef CCDC_MAP_BLOCKS_PER_SM
+#define CCDC_MAP_BLOCKS_PER_SM 3     // resident blocks per SM: bounds the files in flight, i.e. the L2 footprint
 #endif
-constexpr int MAP_THREADS = 256;                 // pass 1: 8 warps share 16 rows
+#ifndef CCDC_MAP_MIN_BLOCKS
+#define CCDC_MAP_MIN_BLOCKS 2        // register budget: 65536 / (256 * MIN_BLOCKS) per thread
+#endif
+#ifndef CCDC_MAP_DEPTH1
+#define CCDC_MAP_DEPTH1 8            // pass 1: 32-column quarters per trip (2 loads each)
+#endif
+#ifndef CCDC_MAP_DEPTH2
+#define CCDC_MAP_DEPTH2 2            // pass 2: 16-row steps per trip (4 loads each)
+#endif
+#ifndef CCDC_MAP_LAG
+#define CCDC_MAP_LAG 4               // pass 2 of file f is handed out after pass 1 of file f + LAG
+#endif
+constexpr int MAP_THREADS = 256;                 // 8 warps
 constexpr int MAP_WARPS = MAP_THREADS / 32;
-constexpr int GRAD_THREADS = 128;                // pass 2: 4 warps x 64 columns
-constexpr int GRAD_WARPS = GRAD_THREADS / 32;
-constexpr int GRAD_COLS = GRAD_WARPS * 64;
+constexpr int GRAD_COLS = MAP_WARPS * 64;        // pass 2: columns per block
+constexpr int WAIT_LIMIT = 1 << 20;              // polls of a file's pass-1 counter before giving up
 
 struct MapParams {
     const uint16_t *x[CCDC_MAX_K];      // node k: [local file][rows][d] bf16
@@ -44,7 +50,10 @@ struct MapParams {
     long long first_job[CCDC_MAX_K + 1];// jobs are (node, local file), node-major
     const uint16_t *w;                  // [d] bf16
     float *u;                           // [jobs][rows] residuals (workspace)
-    long long job0, njobs;              // this wave
+    int *done;                          // [jobs] pass-1 blocks finished per job (workspace, zeroed per call)
+    int *ticket;                        // next work item (workspace, zeroed per call)
+    int *status;                        // set to 1 if a wait ran out (workspace, zeroed per call)
+    long long njobs;
     long long rows, d;
     int K;
 };
@@ -57,49 +66,67 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// 16-byte read-only load with an L2 eviction policy: pass 1 asks L2 to keep X
+// (evict last), pass 2 reads it for the last time (evict first)
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_drop() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint4 load_keep(const uint16_t *ptr, uint64_t policy) {
+    uint4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(ptr), "l"(policy));
+    return v;
+}
+
 __device__ __forceinline__ int node_of_job(const MapParams &p, long long job) {
     int k = 0;
     while (k + 1 < p.K && job >= p.first_job[k + 1]) ++k;
     return k;
 }
 
-// ---- pass 1: u = X w - y for 16 rows of one file per block.
+// ---- pass 1: u = X w - y for 16 rows of one file.
 // The k index of the MMA is a free relabelling of the columns: thread (g, t)
 // of a warp loads 8 consecutive columns of rows g and g+8 with one 16-byte load
 // each and feeds them as k = 2t, 2t+1, 2t+8, 2t+9 of two MMAs; w is placed in
 // column n = 0 of B with the same relabelling (lanes with g = 0), the other
-// columns are zero.
-__global__ void __launch_bounds__(MAP_THREADS)
-k_map_residual(const __grid_constant__ MapParams p) {
-    extern __shared__ __align__(16) uint32_t sh_w[];        // d/2 words: w as bf16 pairs
-    __shared__ float sh_part[MAP_WARPS][16];
-    const long long row_blocks = p.rows / 16;
-    const long long job = p.job0 + blockIdx.x / row_blocks;
-    const long long row0 = (blockIdx.x % row_blocks) * 16;
+// columns are zero.  The 8 warps split the columns; their partial dots are
+// added in warp order.
+template <int QUARTERS>     // 32-column quarters per loop trip: 2 * QUARTERS loads in flight per thread
+__device__ __forceinline__ void residual_block(const MapParams &p, const uint32_t *sh_w, float (*sh_part)[16],
+                                               long long job, long long row0) {
     const int k = node_of_job(p, job);
     const long long file = job - p.first_job[k];
     const uint16_t *X = p.x[k] + (file * p.rows + row0) * p.d;
-
-    for (long long i = threadIdx.x; i < p.d / 8; i += MAP_THREADS)
-        reinterpret_cast<uint4 *>(sh_w)[i] = __ldg(reinterpret_cast<const uint4 *>(p.w) + i);
-    __syncthreads();
-
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int g = lane / 4, t = lane % 4;
     const long long cols_per_warp = p.d / MAP_WARPS;        // a multiple of 64
     const uint16_t *rowA = X + (long long)g * p.d;
     const uint16_t *rowB = X + (long long)(g + 8) * p.d;
+    const uint64_t keep = l2_policy_keep();
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (long long c0 = warp * cols_per_warp; c0 < (warp + 1) * cols_per_warp; c0 += 64) {
+    for (long long c0 = warp * cols_per_warp; c0 < (warp + 1) * cols_per_warp; c0 += 32 * QUARTERS) {
+        uint4 va[QUARTERS], vb[QUARTERS];
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const long long c = c0 + 32 * half + 8 * t;
-            const uint4 va = __ldg(reinterpret_cast<const uint4 *>(rowA + c));
-            const uint4 vb = __ldg(reinterpret_cast<const uint4 *>(rowB + c));
+        for (int q = 0; q < QUARTERS; ++q) {         // all loads of the trip first
+            const long long c = c0 + 32 * q + 8 * t;
+            va[q] = load_keep(rowA + c, keep);
+            vb[q] = load_keep(rowB + c, keep);
+        }
+#pragma unroll
+        for (int q = 0; q < QUARTERS; ++q) {
+            const long long c = c0 + 32 * q + 8 * t;
             uint4 wv = make_uint4(0u, 0u, 0u, 0u);
             if (g == 0) wv = *reinterpret_cast<const uint4 *>(sh_w + c / 2);
-            mma_bf16(acc, va.x, vb.x, va.y, vb.y, wv.x, wv.y);
-            mma_bf16(acc, va.z, vb.z, va.w, vb.w, wv.z, wv.w);
+            mma_bf16(acc, va[q].x, vb[q].x, va[q].y, vb[q].y, wv.x, wv.y);
+            mma_bf16(acc, va[q].z, vb[q].z, va[q].w, vb[q].w, wv.z, wv.w);
         }
     }
     // column n = 0 of the accumulator tile: thread (g, t = 0) holds rows g and g+8
@@ -113,10 +140,13 @@ k_map_residual(const __grid_constant__ MapParams p) {
         for (int wv = 1; wv < MAP_WARPS; ++wv) s += sh_part[wv][threadIdx.x];   // fixed order
         const long long r = row0 + threadIdx.x;
         p.u[job * p.rows + r] = s - p.y[k][file * p.rows + r];
+        __threadfence();                    // the residuals are visible before the job's counter moves
     }
+    __syncthreads();
+    if (threadIdx.x == 0) atomicAdd(p.done + job, 1);
 }
 
-// ---- pass 2: g = X^T u for GRAD_COLS columns of one file per block.
+// ---- pass 2: g = X^T u for GRAD_COLS columns of one file.
 // A (16 x 16): row 0, 1, 2 = the three bf16 terms of u (u = hi + mid + lo to
 // about 2^-25 relative), the other rows zero; k = 16 rows of X.  B (16 x 8):
 // thread (g, t) supplies column n = g for k = 2t, 2t+1, 2t+8, 2t+9, i.e. one
@@ -124,20 +154,16 @@ k_map_residual(const __grid_constant__ MapParams p) {
 // and serves eight MMAs, one per column of its octet, packing two rows into a
 // register with a byte permute.  MMA e therefore produces, at n = g', column
 // j0 + 8 g' + e.
-__global__ void __launch_bounds__(GRAD_THREADS)
-k_map_gradient(const __grid_constant__ MapParams p) {
-    extern __shared__ __align__(16) uint32_t sh_u[];        // [3][rows/2] bf16 pairs: hi, mid, lo
-    const long long col_blocks = (p.d + GRAD_COLS - 1) / GRAD_COLS;
-    const long long job = p.job0 + blockIdx.x / col_blocks;
-    const long long col0 = (blockIdx.x % col_blocks) * GRAD_COLS;
+template <int STEPS>        // 16-row steps per loop trip: 4 * STEPS loads in flight per thread
+__device__ __forceinline__ void gradient_block(const MapParams &p, uint32_t *sh_u, long long job, long long col0) {
     const int k = node_of_job(p, job);
     const long long file = job - p.first_job[k];
     const uint16_t *X = p.x[k] + file * p.rows * p.d;
     const long long half_rows = p.rows / 2;
-
-    for (long long i = threadIdx.x; i < half_rows; i += GRAD_THREADS) {
-        uint32_t packed[3];
-        float v[2] = {p.u[job * p.rows + 2 * i], p.u[job * p.rows + 2 * i + 1]};
+    for (long long i = threadIdx.x; i < half_rows; i += MAP_THREADS) {
+        // written by other blocks of this launch: read through L2, not the SM's L1
+        const float2 v2 = __ldcg(reinterpret_cast<const float2 *>(p.u + job * p.rows) + i);
+        const float v[2] = {v2.x, v2.y};
         uint16_t term[3][2];
         for (int e = 0; e < 2; ++e) {
             float rest = v[e];
@@ -147,65 +173,131 @@ k_map_gradient(const __grid_constant__ MapParams p) {
                 rest = rest - __bfloat162float(h);          // exact in fp32
             }
         }
-        for (int s = 0; s < 3; ++s) packed[s] = (uint32_t)term[s][0] | ((uint32_t)term[s][1] << 16);
-        sh_u[i] = packed[0];
-        sh_u[half_rows + i] = packed[1];
-        sh_u[2 * half_rows + i] = packed[2];
+        for (int s = 0; s < 3; ++s) sh_u[s * half_rows + i] = (uint32_t)term[s][0] | ((uint32_t)term[s][1] << 16);
     }
     __syncthreads();
 
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int g = lane / 4, t = lane % 4;
     const long long j0 = col0 + warp * 64;
-    if (j0 >= p.d) return;
-    const uint16_t *base = X + j0 + 8 * g;
-    float acc[8][4];
+    if (j0 < p.d) {
+        const uint16_t *base = X + j0 + 8 * g;
+        const uint64_t drop = l2_policy_drop();
+        float acc[8][4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
-
-    for (long long i0 = 0; i0 < p.rows; i0 += 16) {
-        const long long r0 = i0 + 2 * t;
-        const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(base + r0 * p.d));
-        const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(base + (r0 + 1) * p.d));
-        const uint4 v2 = __ldg(reinterpret_cast<const uint4 *>(base + (r0 + 8) * p.d));
-        const uint4 v3 = __ldg(reinterpret_cast<const uint4 *>(base + (r0 + 9) * p.d));
-        uint32_t a0 = 0u, a2 = 0u;
-        if (g < 3) {
-            a0 = sh_u[g * half_rows + r0 / 2];
-            a2 = sh_u[g * half_rows + (r0 + 8) / 2];
+        for (int e = 0; e < 8; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
+        for (long long i0 = 0; i0 < p.rows; i0 += 16 * STEPS) {
+            uint4 v[STEPS][4];
+#pragma unroll
+            for (int h = 0; h < STEPS; ++h) {            // all loads of the trip first
+                const long long r0 = i0 + 16 * h + 2 * t;
+                v[h][0] = load_keep(base + r0 * p.d, drop);
+                v[h][1] = load_keep(base + (r0 + 1) * p.d, drop);
+                v[h][2] = load_keep(base + (r0 + 8) * p.d, drop);
+                v[h][3] = load_keep(base + (r0 + 9) * p.d, drop);
+            }
+#pragma unroll
+            for (int h = 0; h < STEPS; ++h) {
+                const long long r0 = i0 + 16 * h + 2 * t;
+                uint32_t a0 = 0u, a2 = 0u;
+                if (g < 3) {
+                    a0 = sh_u[g * half_rows + r0 / 2];
+                    a2 = sh_u[g * half_rows + (r0 + 8) / 2];
+                }
+                const uint32_t w0[4] = {v[h][0].x, v[h][0].y, v[h][0].z, v[h][0].w};
+                const uint32_t w1[4] = {v[h][1].x, v[h][1].y, v[h][1].z, v[h][1].w};
+                const uint32_t w2[4] = {v[h][2].x, v[h][2].y, v[h][2].z, v[h][2].w};
+                const uint32_t w3[4] = {v[h][3].x, v[h][3].y, v[h][3].z, v[h][3].w};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;   // high or low halves of both words
+                    const uint32_t b0 = __byte_perm(w0[e / 2], w1[e / 2], sel);
+                    const uint32_t b1 = __byte_perm(w2[e / 2], w3[e / 2], sel);
+                    mma_bf16(acc[e], a0, 0u, a2, 0u, b0, b1);
+                }
+            }
         }
-        const uint32_t w0[4] = {v0.x, v0.y, v0.z, v0.w}, w1[4] = {v1.x, v1.y, v1.z, v1.w};
-        const uint32_t w2[4] = {v2.x, v2.y, v2.z, v2.w}, w3[4] = {v3.x, v3.y, v3.z, v3.w};
+        // rows 0, 1, 2 of the accumulator tiles live in lanes g = 0, 1, 2 (same t):
+        // g = (hi + mid) + lo, then lanes g = 0 write 16 consecutive outputs
+        uint32_t *out = p.part[k] + file * p.d;
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;       // high or low halves of both words
-            const uint32_t b0 = __byte_perm(w0[e / 2], w1[e / 2], sel);
-            const uint32_t b1 = __byte_perm(w2[e / 2], w3[e / 2], sel);
-            mma_bf16(acc[e], a0, 0u, a2, 0u, b0, b1);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                const float hi = acc[e][c];
+                const float mid = __shfl_down_sync(0xffffffffu, hi, 4);
+                const float lo = __shfl_down_sync(0xffffffffu, hi, 8);
+                acc[e][c] = (hi + mid) + lo;
+            }
+        }
+        if (g == 0) {
+            // column of acc[e][c] = j0 + 8 * (2t + c) + e
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                float4 lo4 = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
+                float4 hi4 = make_float4(acc[4][c], acc[5][c], acc[6][c], acc[7][c]);
+                float *dst = reinterpret_cast<float *>(out) + j0 + 8 * (2 * t + c);
+                *reinterpret_cast<float4 *>(dst) = lo4;
+                *reinterpret_cast<float4 *>(dst + 4) = hi4;
+            }
         }
     }
-    // rows 0, 1, 2 of the accumulator tiles live in lanes g = 0, 1, 2 (same t):
-    // g = (hi + mid) + lo, then lanes g = 0 write 16 consecutive outputs
-    uint32_t *out = p.part[k] + file * p.d;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            const float hi = acc[e][c];
-            const float mid = __shfl_down_sync(0xffffffffu, hi, 4);
-            const float lo = __shfl_down_sync(0xffffffffu, hi, 8);
-            acc[e][c] = (hi + mid) + lo;
-        }
-    }
-    if (g == 0) {
-        // column of acc[e][c] = j0 + 8 * (2t + c) + e
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-            float4 lo4 = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
-            float4 hi4 = make_float4(acc[4][c], acc[5][c], acc[6][c], acc[7][c]);
-            float *dst = reinterpret_cast<float *>(out) + j0 + 8 * (2 * t + c);
-            *reinterpret_cast<float4 *>(dst) = lo4;
-            *reinterpret_cast<float4 *>(dst + 4) = hi4;
+}
+
+// ---- both passes in one launch, so that pass 2 finds the file in L2.
+// Work items are handed out in order through an atomic ticket: per file, its
+// n1 pass-1 blocks (16 rows each), then the n2 pass-2 blocks (512 columns each)
+// of the file LAG places earlier.  With 148 x 3 blocks resident only a handful
+// of files (a few tens of MB of X) are between their two passes at any time,
+// so the second read of X is served by L2 and DRAM sees X once.
+// A pass-2 item waits until the file's pass-1 counter is complete.  Those
+// pass-1 items carry smaller tickets, so they were taken by blocks that are
+// already running and that wait on nothing: the wait always ends.  It is
+// bounded all the same; if it ever ran out the block records that in `status`
+// and goes on (the file's output is then wrong and ccdc_map_status says so).
+__global__ void __launch_bounds__(MAP_THREADS, CCDC_MAP_MIN_BLOCKS)
+k_map(const __grid_constant__ MapParams p) {
+    extern __shared__ __align__(16) uint32_t sh[];
+    uint32_t *sh_w = sh;                        // d/2 words: w as bf16 pairs
+    uint32_t *sh_u = sh + p.d / 2;              // 3 * rows/2 words: u as hi / mid / lo bf16 pairs
+    __shared__ float sh_part[MAP_WARPS][16];
+    __shared__ long long sh_ticket;
+
+    for (long long i = threadIdx.x; i < p.d / 8; i += MAP_THREADS)
+        reinterpret_cast<uint4 *>(sh_w)[i] = __ldg(reinterpret_cast<const uint4 *>(p.w) + i);
+
+    const long long n1 = p.rows / 16, n2 = (p.d + GRAD_COLS - 1) / GRAD_COLS, per = n1 + n2;
+    const long long total = (p.njobs + CCDC_MAP_LAG) * per;
+    // deeper load pipelines when the shape divides evenly
+    const bool deep1 = (p.d / MAP_WARPS) % (32 * CCDC_MAP_DEPTH1) == 0;
+    const bool deep2 = p.rows % (16 * CCDC_MAP_DEPTH2) == 0;
+    for (;;) {
+        __syncthreads();                        // sh_ticket, sh_u and sh_part are free again
+        if (threadIdx.x == 0) sh_ticket = atomicAdd(p.ticket, 1);
+        __syncthreads();
+        const long long tk = sh_ticket;
+        if (tk >= total) break;
+        const long long step = tk / per, slot = tk - step * per;
+        if (slot < n1) {
+            if (step < p.njobs) {
+                if (deep1) residual_block<CCDC_MAP_DEPTH1>(p, sh_w, sh_part, step, slot * 16);
+                else residual_block<2>(p, sh_w, sh_part, step, slot * 16);
+            }
+        } else {
+            const long long job = step - CCDC_MAP_LAG;
+            if (job < 0) continue;
+            if (threadIdx.x == 0) {
+                const volatile int *done = p.done + job;
+                int polls = 0;
+                while (*done < (int)n1) {
+                    if (++polls > WAIT_LIMIT) { atomicExch(p.status, 1); break; }
+                    __nanosleep(100);
+                }
+                __threadfence();
+            }
+            __syncthreads();
+            if (deep2) gradient_block<CCDC_MAP_DEPTH2>(p, sh_u, job, (slot - n1) * GRAD_COLS);
+            else gradient_block<1>(p, sh_u, job, (slot - n1) * GRAD_COLS);
         }
     }
 }
@@ -216,13 +308,19 @@ long long total_jobs(const ccdc_plan_s &P) {
     return n;
 }
 
+// workspace layout: residuals [jobs][rows] fp32, then (256-byte aligned) the
+// pass-1 counters [jobs], the ticket and the status word
+size_t residual_bytes(long long jobs, long long rows) { return ((size_t)(jobs * rows) * 4 + 255) / 256 * 256; }
+size_t control_bytes(long long jobs) { return ((size_t)(jobs + 2) * 4 + 255) / 256 * 256; }
+
 }  // namespace
 
 extern "C" {
 
 size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows) {
     if (!plan || rows <= 0) return 0;
-    return (size_t)(total_jobs(*plan) * rows) * sizeof(float);
+    const long long jobs = total_jobs(*plan);
+    return residual_bytes(jobs, rows) + control_bytes(jobs);
 }
 
 int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
@@ -245,31 +343,43 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
         mp.part[k] = static_cast<uint32_t *>(part[k]);
     }
     if ((reinterpret_cast<uintptr_t>(w) & 15u) || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return CCDC_EINVAL;
+    const long long njobs = mp.first_job[P.K];
+    if (njobs * (rows / 16 + (d + GRAD_COLS - 1) / GRAD_COLS) > 0x3fffffffLL) return CCDC_ESIZE;   // tickets are ints
     mp.w = static_cast<const uint16_t *>(w);
     mp.u = static_cast<float *>(workspace);
-    mp.rows = rows; mp.d = d; mp.K = P.K;
-    const long long njobs = mp.first_job[P.K];
+    int *control = reinterpret_cast<int *>(static_cast<char *>(workspace) + residual_bytes(njobs, rows));
+    mp.done = control;
+    mp.ticket = control + njobs;
+    mp.status = control + njobs + 1;
+    mp.njobs = njobs; mp.rows = rows; mp.d = d; mp.K = P.K;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const long long file_bytes = rows * d * 2;
-    const long long wave = CCDC_MAP_WAVE_MB > 0 ? std::max(1LL, ((long long)CCDC_MAP_WAVE_MB << 20) / file_bytes)
-                                                : std::max(1LL, njobs);
-    const size_t smem1 = (size_t)d * 2, smem2 = (size_t)rows * 6;
-    if (smem1 > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(k_map_residual, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    cudaError_t e = cudaMemsetAsync(control, 0, control_bytes(njobs), st);
+    if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+    const size_t smem = (size_t)d * 2 + (size_t)rows * 6;
+    if (smem > 32 * 1024) {
+        e = cudaFuncSetAttribute(k_map, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
     }
-    const long long col_blocks = (d + GRAD_COLS - 1) / GRAD_COLS;
-    for (long long j0 = 0; j0 < njobs; j0 += wave) {
-        mp.job0 = j0;
-        mp.njobs = std::min(wave, njobs - j0);
-        k_map_residual<<<(unsigned)(mp.njobs * (rows / 16)), MAP_THREADS, smem1, st>>>(mp);
-        ccdc_internal_count_launch();
-        k_map_gradient<<<(unsigned)(mp.njobs * col_blocks), GRAD_THREADS, smem2, st>>>(mp);
-        ccdc_internal_count_launch();
-        cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
-    }
-    return CCDC_OK;
+    int dev = 0, sms = 0, per_sm = 0;
+    e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_map, MAP_THREADS, smem);
+    if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+    per_sm = std::max(1, std::min(per_sm, CCDC_MAP_BLOCKS_PER_SM));
+    k_map<<<(unsigned)(sms * per_sm), MAP_THREADS, smem, st>>>(mp);
+    ccdc_internal_count_launch();
+    e = cudaGetLastError();
+    return e == cudaSuccess ? CCDC_OK : ccdc_internal_cuda_fail((int)e);
+}
+
+int ccdc_map_status(const ccdc_plan_t *plan, long long rows, const void *workspace) {
+    if (!plan || !workspace || rows <= 0) return CCDC_EINVAL;
+    const long long jobs = total_jobs(*plan);
+    const char *status = static_cast<const char *>(workspace) + residual_bytes(jobs, rows) + (size_t)(jobs + 1) * 4;
+    int word = 0;
+    cudaError_t e = cudaMemcpy(&word, status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+    return word == 0 ? CCDC_OK : CCDC_ESTATE;
 }
 
 }  // extern "C"
