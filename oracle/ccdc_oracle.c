@@ -667,3 +667,91 @@ int64_t oracle_bits_plain_cdc(const ccdc_oracle *o)
 
 /* files stored at node k (storage constraint of Section III) */
 int64_t oracle_node_num_files(const ccdc_oracle *o, int k) { return o->nlocal[k] * o->b; }
+
+/* ------------------------------------------------------------------ */
+/* Compression-only scheme (Appendix, "Communication Load of the compression
+ * scheme"), one job.  The files are cut into m = ceil(1/mu) batches: the first
+ * m-1 hold mu*N files each, the last one the rest; node k stores batch k mod m
+ * (0-based).  For every function of node k and every batch t it does not store,
+ * one node that stores batch t pre-combines the batch for that function and
+ * unicasts the packet to k; k adds the m-1 packets to its own batch sum.
+ * The paper leaves the choice of the sender open; here it is the first node
+ * after k, cyclically, that stores batch t.
+ *
+ * v     [N][Q][B] words, mu = r/K (K | r*N required)
+ * out   [Q][B]
+ * recv  [K][m-1][len]: packets node k received, batches ascending
+ * returns the number of bits sent (every unicast counted once, Definition 1),
+ * or -1 on invalid parameters / memory.                                   */
+int64_t oracle_compression_run(int K, int r, int64_t N, int Q, int64_t B, int dtype,
+                               const uint32_t *v, uint32_t *out, uint32_t *recv,
+                               int64_t *files_at_node /* [K] */)
+{
+    if (K < 2 || r < 1 || r > K - 1 || N < K || Q % K != 0 || B < 1) return -1;
+    if ((r * N) % K != 0) return -1;
+    const int m = (K + r - 1) / r;                   /* ceil(1/mu) */
+    const int64_t full = r * N / K;                  /* mu*N files in the first m-1 batches */
+    const int64_t last = N - (int64_t)(m - 1) * full;
+    if (last < 1) return -1;
+    const int per = Q / K;
+    const int64_t len = (int64_t)per * B, row = (int64_t)Q * B;
+    uint32_t **mem = (uint32_t **)calloc((size_t)K, sizeof(uint32_t *));
+    if (!mem) return -1;
+    int64_t bits = 0;
+    /* placement: node k holds a private copy of batch k mod m */
+    for (int k = 0; k < K; ++k) {
+        const int t = k % m;
+        const int64_t nf = t == m - 1 ? last : full;
+        mem[k] = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)(nf * row));
+        if (!mem[k]) { bits = -1; goto done; }
+        memcpy(mem[k], v + (int64_t)t * full * row, sizeof(uint32_t) * (size_t)(nf * row));
+        if (files_at_node) files_at_node[k] = nf;
+    }
+    /* shuffle: unicast of pre-combined packets */
+    for (int k = 0; k < K; ++k) {
+        int slot = 0;
+        for (int t = 0; t < m; ++t) {
+            if (t == k % m) continue;
+            int ks = (k + 1) % K;
+            while (ks % m != t) ks = (ks + 1) % K;   /* first node after k that stores batch t */
+            const int64_t nf = t == m - 1 ? last : full;
+            uint32_t *pkt = recv + ((int64_t)k * (m - 1) + slot) * len;
+            for (int c = 0; c < per; ++c)
+                for (int64_t e = 0; e < B; ++e) {
+                    const int q = k * per + c;
+                    uint32_t acc = mem[ks][(int64_t)q * B + e];
+                    for (int64_t f = 1; f < nf; ++f)
+                        acc = add_words(dtype, acc, mem[ks][(f * Q + q) * B + e]);
+                    pkt[(int64_t)c * B + e] = acc;
+                }
+            bits += 32 * len;
+            ++slot;
+        }
+    }
+    /* reduce at node k: batches ascending, own batch from own memory */
+    for (int k = 0; k < K; ++k)
+        for (int c = 0; c < per; ++c)
+            for (int64_t e = 0; e < B; ++e) {
+                const int q = k * per + c;
+                uint32_t acc = 0u;
+                int slot = 0;
+                for (int t = 0; t < m; ++t) {
+                    uint32_t term;
+                    if (t == k % m) {
+                        const int64_t nf = t == m - 1 ? last : full;
+                        term = mem[k][(int64_t)q * B + e];
+                        for (int64_t f = 1; f < nf; ++f)
+                            term = add_words(dtype, term, mem[k][(f * Q + q) * B + e]);
+                    } else {
+                        term = recv[((int64_t)k * (m - 1) + slot) * len + (int64_t)c * B + e];
+                        ++slot;
+                    }
+                    acc = add_words(dtype, acc, term);
+                }
+                out[(int64_t)q * B + e] = acc;
+            }
+done:
+    for (int k = 0; k < K; ++k) free(mem[k]);
+    free(mem);
+    return bits;
+}

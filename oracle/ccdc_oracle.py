@@ -81,6 +81,7 @@ def _load():
         "oracle_bits_uncoded": (L, [P]),
         "oracle_bits_combining": (L, [P]),
         "oracle_bits_plain_cdc": (L, [P]),
+        "oracle_compression_run": (L, [I, I, L, I, L, I, P, P, P, P]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -244,6 +245,27 @@ class Oracle:
     @property
     def bits_plain_cdc(self):
         return _load().oracle_bits_plain_cdc(self._h)
+
+
+def compression_only(K, r, N, Q, B, dtype, v):
+    """The compression-only scheme of the paper's appendix (one job, mu = r/K).
+
+    Returns ``(out [Q][B], recv [K][m-1][len], bits, files_at_node [K])``.
+    """
+    lib = _load()
+    dt = {"int32": I32, "float32": F32}[dtype]
+    npdt = np.int32 if dt == I32 else np.float32
+    v = np.ascontiguousarray(v)
+    assert v.dtype == npdt and v.shape == (N, Q, B)
+    m = -(-K // r)
+    ln = (Q // K) * B
+    out = np.zeros((Q, B), dtype=np.uint32)
+    recv = np.zeros((K, m - 1, ln), dtype=np.uint32)
+    files = np.zeros(K, dtype=np.int64)
+    bits = lib.oracle_compression_run(K, r, N, Q, B, dt, _ptr(v), _ptr(out), _ptr(recv), _ptr(files))
+    if bits < 0:
+        raise ValueError(f"invalid parameters K={K} r={r} N={N} Q={Q} B={B}")
+    return out.view(npdt), recv, bits, files.tolist()
 
 
 def map_linear_regression(X: np.ndarray, w: np.ndarray, y: np.ndarray, Q: int) -> np.ndarray:

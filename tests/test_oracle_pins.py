@@ -501,3 +501,48 @@ def test_map_linear_regression_is_the_gradient():
         e = np.zeros(d); e[j] = h
         fd = (f(w.astype(np.float64) + e) - f(w.astype(np.float64) - e)) / (2 * h)
         assert abs(fd - g[j]) <= 1e-5 * max(1.0, abs(g[j]))
+
+
+# ------------------------------------------------ compression-only comparator
+@pytest.mark.parametrize("K,r,N", [(4, 2, 8), (6, 2, 12), (6, 1, 12), (5, 2, 10), (7, 3, 14), (8, 3, 16),
+                                   (6, 4, 12), (10, 3, 20), (5, 4, 10)])
+def test_compression_only_load_and_result(K, r, N):
+    """Appendix: with mu = r/K the compression-only scheme sends ceil(1/mu)-1 packets
+    of one value per function, L = ceil(1/mu)-1 (which is 1 for mu >= 1/2), every
+    node stores at most mu*N files and every output is the direct sum of Eq. (1)."""
+    from oracle.ccdc_oracle import compression_only
+
+    Q, B = 2 * K, 6
+    for dt in ("int32", "float32"):
+        v = values_numpy(N, Q, B, dt, seed=K + r)
+        out, recv, bits, files = compression_only(K, r, N, Q, B, dt, v)
+        mu = Fraction(r, K)
+        m = -(-K // r)
+        expect_L = (-(-1 // mu) - 1) if mu < Fraction(1, 2) else 1
+        assert m - 1 == expect_L or mu >= Fraction(1, 2)
+        assert Fraction(bits, Q * 32 * B) == m - 1
+        if mu <= Fraction(1, 2):
+            assert Fraction(bits, Q * 32 * B) == -(-1 // mu) - 1
+        else:
+            assert Fraction(bits, Q * 32 * B) == 1
+        assert all(f <= mu * N for f in files) and recv.shape == (K, m - 1, (Q // K) * B)
+        if dt == "int32":
+            expect = (v.astype(np.int64).sum(axis=0) & 0xFFFFFFFF).astype(np.uint32).view(np.int32)
+            assert np.array_equal(out, expect)
+        else:
+            s64 = v.astype(np.float64).sum(axis=0)
+            a64 = np.abs(v.astype(np.float64)).sum(axis=0)
+            assert np.all(np.abs(out - s64) <= N * 2.0 ** -24 * a64)
+
+
+def test_compression_only_running_example(golden_dir):
+    """Remark after the K=4 example: combining alone sends 4 pre-combined packets,
+    one for each node, per job: L = 4/4 = 1."""
+    from oracle.ccdc_oracle import compression_only
+
+    rows = read_golden(golden_dir / "running_example_k4.txt")
+    K, r, N, Q = (int(golden_scalar(rows, k)) for k in ("K", "r", "N", "Q"))
+    B = 4
+    out, recv, bits, files = compression_only(K, r, N, Q, B, "int32", values_numpy(N, Q, B, "int32"))
+    assert recv.shape[0] * recv.shape[1] == 4
+    assert Fraction(bits, Q * 32 * B) == golden_scalar(rows, "load_compression")
