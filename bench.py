@@ -388,6 +388,66 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_compression(args, w):
+    """Comparator: the appendix's compression-only shuffle on the same workload shape
+    (unicast of pre-combined packets, no coding).  Same JSON contract; `config.scheme`
+    says what ran."""
+    import torch
+
+    from paper_1805_01993_b200 import build as lib_build
+    from paper_1805_01993_b200 import ccdc
+
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise RuntimeError("the comparator runs on one GPU")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    lib_build.build_library()
+    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, compression=True)
+    plan.upload()
+    part = plan.alloc_partitions(dev)
+    plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=DEFAULT_SEED, std=w.std))
+    recv = plan.alloc_decoded(dev)
+    out = plan.alloc(plan.out_bytes, dev)
+    m = plan.num_batches
+    ln = plan.packet_elems * 4
+    nfiles = [len(plan.node_files(k)) for k in range(w.K)]
+    full, last = plan.files_per_batch, w.N - (m - 1) * plan.files_per_batch
+    sent = sum((last if t == m - 1 else full) for k in range(w.K) for t in range(m) if t != k % m)
+    iv_read = (sent + sum(nfiles)) * ln                       # batches pre-combined for others + own batch
+    total = iv_read + 2 * w.K * (m - 1) * ln + plan.out_bytes   # + packets written and read + outputs
+    stream = torch.cuda.current_stream()
+    for _ in range(args.warmup):
+        plan.compression_shuffle(part, recv, out)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    time.sleep(0.3)
+    l0 = ccdc.num_kernel_launches()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(args.steps):
+        plan.compression_shuffle(part, recv, out)
+    b.record(stream)
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / args.steps
+    peaks_file = ROOT / "MEASURED_PEAKS.json"
+    peak = json.loads(peaks_file.read_text())["hbm_gbs"] if peaks_file.exists() else 6650.0
+    print(json.dumps({
+        "metric": METRIC, "value": iv_read / (ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if w.dtype == "float32" else "i32", "data": "synthetic",
+        "config": {"workload": w.name, "scheme": "compression-only (appendix), comparator", "K": w.K, "r": w.r,
+                   "N": w.N, "Q": w.Q, "B": w.B, "batches": m, "unicast_bits": plan.coded_bits,
+                   "load_per_QT": plan.coded_bits / (w.Q * 32 * w.B), "iv_bytes_per_step": iv_read,
+                   "algorithmic_bytes_per_step": total},
+        "roofline": {"bound": "hbm", "kernel": "k_gather(combine)+k_reduce", "achieved": total / (ms * 1e-3) / 1e9,
+                     "peak": peak, "unit": "GB/s", "frac": total / (ms * 1e-3) / 1e9 / peak, "traffic": None},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": ccdc.num_kernel_launches() - l0,
+        "clocks": sampler.stop(),
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -397,6 +457,8 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(CONFIGS))
     ap.add_argument("--value-elems", type=int, default=0,
                     help="shorten every value to this many elements (profiling captures on a small case)")
+    ap.add_argument("--scheme", choices=["ccdc", "compression"], default="ccdc",
+                    help="compression = the appendix's compression-only shuffle, as a comparator")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave out the oracle timing leg")
     args = ap.parse_args()
@@ -405,6 +467,8 @@ def main():
         w = w.scaled(args.value_elems)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.scheme == "compression":
+        run_compression(args, w)
     else:
         run_ours(args, w)
 

@@ -92,6 +92,20 @@ typedef enum {
  * Host only: no CUDA call is made.  Destroy with ccdc_plan_destroy. */
 int  ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
 int  ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
+/* ccdc_plan_compression: the compression-only scheme of the paper's appendix
+ * ("Communication Load of the compression scheme"), kept as a measured
+ * comparator.  One job, mu = r/K: the files are cut into m = ceil(K/r) batches,
+ * the first m-1 of mu*N files and the last of the rest; node k stores batch
+ * k mod m (so its partition is [file in batch][q][B] with ccdc_plan_batch_files
+ * files); for every batch t it lacks, node k is sent ONE pre-combined packet of
+ * its Q/K functions by the first node after k, cyclically, that stores batch t
+ * (the paper leaves the sender open).  No coding: only ccdc_compression_shuffle
+ * and ccdc_reduce accept such a plan, the coded steps return CCDC_ESTATE.
+ * ccdc_plan_coded_bits is then the unicast bit count K*(m-1)*32*len, i.e. the
+ * load ceil(1/mu)-1 of Eq. (2).   requires additionally K | r*N.
+ * Queries: ccdc_plan_num_batches = m, ccdc_plan_num_groups = 0, holders of a
+ * batch are reported in r slots padded with -1. */
+int  ccdc_plan_compression(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
 void ccdc_plan_destroy(ccdc_plan_t *plan);
 
 /* Copies the schedule tables to the current device (cudaMalloc + cudaMemcpy,
@@ -106,6 +120,8 @@ long long ccdc_plan_num_jobs(const ccdc_plan_t *plan);        /* J */
 long long ccdc_plan_num_batches(const ccdc_plan_t *plan);     /* over all jobs */
 long long ccdc_plan_num_groups(const ccdc_plan_t *plan);      /* multicast rounds: C(K,r+1) per job batch set */
 long long ccdc_plan_files_per_batch(const ccdc_plan_t *plan); /* b */
+long long ccdc_plan_batch_files(const ccdc_plan_t *plan, long long p); /* files in batch p (differs from b only
+                                                                           for the last batch of a compression plan) */
 long long ccdc_plan_packet_elems(const ccdc_plan_t *plan);    /* len = (Q/K)*B */
 long long ccdc_plan_segment_elems(const ccdc_plan_t *plan);   /* s = ceil(len/r) */
 long long ccdc_plan_coded_row_elems(const ccdc_plan_t *plan); /* s_pad */
@@ -210,6 +226,16 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
                        void *workspace, void *stream);
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out,
                  void *workspace, void *stream);
+
+/* The appendix's compression-only shuffle (comparator; plans from
+ * ccdc_plan_compression only, else CCDC_ESTATE).  recv: device pointer array,
+ * recv[k] = ccdc_decoded_bytes(plan, k) = the m-1 packets node k receives,
+ * batches ascending.  Launch 1: every packet = sum over the sender's batch of
+ * the receiver's Q/K values (files ascending, starting from the first file's
+ * value), written to the receiver's buffer.  Launch 2: Eq. (1): batches
+ * ascending, the node's own batch from its partition, the others from recv. */
+int ccdc_compression_shuffle(ccdc_plan_t *plan, const void *const *part, void *const *recv, void *out,
+                             void *stream);
 
 /* ccdc_shuffle on Map results that live in HOST memory (Section III: the
  * Shuffle phase starts from each node's local Map results and ends with the

@@ -27,12 +27,14 @@ _PP = ctypes.POINTER(ctypes.c_void_p)
 SIGNATURES = {
     "ccdc_plan": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_jobs": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
+    "ccdc_plan_compression": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_destroy": (None, [_P]),
     "ccdc_plan_upload": (_I, [_P]),
     "ccdc_plan_num_jobs": (_LL, [_P]),
     "ccdc_plan_num_batches": (_LL, [_P]),
     "ccdc_plan_num_groups": (_LL, [_P]),
     "ccdc_plan_files_per_batch": (_LL, [_P]),
+    "ccdc_plan_batch_files": (_LL, [_P, _LL]),
     "ccdc_plan_packet_elems": (_LL, [_P]),
     "ccdc_plan_segment_elems": (_LL, [_P]),
     "ccdc_plan_coded_row_elems": (_LL, [_P]),
@@ -60,6 +62,7 @@ SIGNATURES = {
     "ccdc_shuffle": (_I, [_P, _PP, _P, _P, _P, _P]),
     "ccdc_static_scratch_bytes": (_SZ, []),
     "ccdc_decode_reduce_static": (_I, [_P, _PP, _P, _P, _P]),
+    "ccdc_compression_shuffle": (_I, [_P, _PP, _PP, _P, _P]),
     "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
     "ccdc_strerror": (ctypes.c_char_p, [_I]),
     "ccdc_last_cuda_error": (_I, []),
@@ -112,12 +115,12 @@ def _stream_handle(stream):
 class Plan:
     """``ccdc_plan`` / ``ccdc_plan_jobs`` plus the step calls on torch tensors."""
 
-    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False):
+    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False, compression: bool = False):
         self.K, self.r, self.N, self.Q, self.B = K, r, N, Q, B
         self.dtype = {"int32": I32, "float32": F32, I32: I32, F32: F32}[dtype]
         self.jobs = jobs
         h = ctypes.c_void_p()
-        fn = lib().ccdc_plan_jobs if jobs else lib().ccdc_plan
+        fn = lib().ccdc_plan_compression if compression else lib().ccdc_plan_jobs if jobs else lib().ccdc_plan
         self._h = None
         _check(fn(K, r, N, Q, B, self.dtype, ctypes.byref(h)), "ccdc_plan")
         self._h = h
@@ -140,13 +143,13 @@ class Plan:
     def batch_of_file(self, n):
         out = (ctypes.c_int * self.r)()
         _check(lib().ccdc_plan_batch_of_file(self._h, n, out), "ccdc_plan_batch_of_file")
-        return list(out)
+        return [k for k in out if k >= 0]
 
     def batch(self, p):
         nodes = (ctypes.c_int * self.r)()
         f0, job = ctypes.c_longlong(), ctypes.c_longlong()
         _check(lib().ccdc_plan_batch(self._h, p, nodes, ctypes.byref(f0), ctypes.byref(job)), "ccdc_plan_batch")
-        return list(nodes), f0.value, job.value
+        return [n for n in nodes if n >= 0], f0.value, job.value
 
     def group(self, g):
         out = (ctypes.c_int * (self.r + 1))()
@@ -190,7 +193,7 @@ class Plan:
         files = []
         for p in self.node_batches(k):
             _, f0, _ = self.batch(p)
-            files.extend(range(f0, f0 + self.files_per_batch))
+            files.extend(range(f0, f0 + lib().ccdc_plan_batch_files(self._h, p)))
         return files
 
     # ---- device buffers (torch is the allocator) --------------------------
@@ -286,6 +289,10 @@ class Plan:
         ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None
         _check(lib().ccdc_decode_reduce(self._h, _ptr_array(part), coded.data_ptr(), out.data_ptr(), ws,
                                         _stream_handle(stream)), "ccdc_decode_reduce")
+
+    def compression_shuffle(self, part, recv, out, stream=None):
+        _check(lib().ccdc_compression_shuffle(self._h, _ptr_array(part), _ptr_array(recv), out.data_ptr(),
+                                              _stream_handle(stream)), "ccdc_compression_shuffle")
 
     def shuffle_host(self, host_part, host_out, part, coded, out, workspace=None, stream=None):
         """``host_part`` / ``host_out``: CPU tensors (pinned for asynchronous copies)."""

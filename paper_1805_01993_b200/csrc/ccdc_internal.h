@@ -46,6 +46,7 @@ struct ccdc_row {
     long long dst_off;
     long long n;
     long long coded_off;
+    long long nf;           // files summed per operand; 0 = the plan's files per batch
 };
 
 // A table of gather rows with a fixed number of operands per row.
@@ -62,6 +63,8 @@ struct ccdc_gather_table {
 struct ccdc_plan_s {
     int K = 0, r = 0, Q = 0, dtype = 0;
     bool jobs_mode = false;
+    bool compression_mode = false;  // the appendix's compression-only comparator (no coding)
+    std::vector<long long> node_nfiles;     // [K] files stored at node k
     long long N = 0, B = 0, J = 1;
     long long b = 0;          // files per batch
     long long len = 0;        // (Q/K)*B

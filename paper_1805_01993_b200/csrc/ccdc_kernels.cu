@@ -183,10 +183,11 @@ k_gather(const __grid_constant__ GatherParams p) {
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
     const int a0 = R.coded_off >= 0 ? -1 : 0;
+    const int nb = R.nf > 0 ? (int)R.nf : p.b;       // files summed per operand
     const long long tj = (long long)threadIdx.x * VEC;
 
     auto advance = [&](GatherCursor &c) {
-        if (c.a >= 0 && ++c.f < p.b) return;
+        if (c.a >= 0 && ++c.f < nb) return;
         c.f = 0;
         if (++c.a >= p.na) { c.a = a0; c.base += TILE; }
     };
@@ -219,7 +220,7 @@ k_gather(const __grid_constant__ GatherParams p) {
         if (ic.base < end) { issue(ic, stage == 0 ? STAGES - 1 : stage - 1); advance(ic); }
         async_commit();
         async_wait<STAGES - 1>();
-        const bool last_file = cc.a < 0 || cc.f == p.b - 1;
+        const bool last_file = cc.a < 0 || cc.f == nb - 1;
         const bool last_of_tile = last_file && cc.a == p.na - 1;
 #pragma unroll
         for (int u = 0; u < GUNROLL; ++u) {
@@ -374,7 +375,8 @@ k_reduce(const __grid_constant__ ReduceParams p) {
     Words<VEC> acc = zero_words<VEC>();
     for (long long t = 0; t < p.nterm; ++t) {
         const ccdc_ref E = terms[t];
-        Words<VEC> v = E.vl == 0 ? batch_sum<VEC, F32>(p.part[k], E.off, j, p.len, p.b, p.file_stride)
+        Words<VEC> v = E.vl <= 0 ? batch_sum<VEC, F32>(p.part[k], E.off, j, p.len, E.vl < 0 ? (int)-E.vl : p.b,
+                                                       p.file_stride)
                                  : load_words<VEC>(p.decoded[k] + E.off + j);
         add_into<VEC, F32>(acc, v);
     }
@@ -523,6 +525,7 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
 }
 
 int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packets, void *stream) {
+    if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
     if (rc == CCDC_OK) rc = check_ptr_array(*plan, (const void *const *)packets, has_part);
@@ -533,6 +536,7 @@ int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packet
 }
 
 int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void *stream) {
+    if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, packets, has_part);
     if (rc == CCDC_OK) rc = ensure_device(plan);
@@ -543,6 +547,7 @@ int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void
 
 int ccdc_decode(ccdc_plan_t *plan, const void *const *packets, const void *coded, void *const *decoded,
                 void *stream) {
+    if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, packets, has_part);
     if (rc == CCDC_OK) rc = check_ptr_array(*plan, (const void *const *)decoded, has_decoded);
@@ -583,6 +588,7 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
 }
 
 int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, void *stream) {
+    if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
     if (rc == CCDC_OK) rc = ensure_device(plan);
@@ -593,6 +599,7 @@ int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, v
 
 int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
                        void *workspace, void *stream) {
+    if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
     if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
@@ -639,6 +646,21 @@ int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *
     int rc = ccdc_encode_fused(plan, part, coded, stream);
     if (rc != CCDC_OK) return rc;
     return ccdc_decode_reduce(plan, part, coded, out, workspace, stream);
+}
+
+int ccdc_compression_shuffle(ccdc_plan_t *plan, const void *const *part, void *const *recv, void *out,
+                             void *stream) {
+    if (!plan || !out || !aligned16(out)) return CCDC_EINVAL;
+    if (!plan->compression_mode) return CCDC_ESTATE;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = check_ptr_array(*plan, (const void *const *)recv, has_decoded);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    // unicast: the sender's pre-combined packet lands in the receiver's buffer
+    rc = launch_gather(*plan, plan->cmb, part, recv, nullptr, nullptr, (int)plan->b, plan->row_elems,
+                       static_cast<cudaStream_t>(stream));
+    if (rc != CCDC_OK) return rc;
+    return ccdc_reduce(plan, part, (const void *const *)recv, out, stream);
 }
 
 int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *host_out, void *const *dev_part,

@@ -304,7 +304,7 @@ k_map(const __grid_constant__ MapParams p) {
 
 long long total_jobs(const ccdc_plan_s &P) {
     long long n = 0;
-    for (int k = 0; k < P.K; ++k) n += P.nlocal[k] * P.b;
+    for (int k = 0; k < P.K; ++k) n += P.node_nfiles[k];
     return n;
 }
 
@@ -327,13 +327,13 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
              long long rows, void *const *part, void *workspace, void *stream) {
     if (!plan || !files_x || !files_y || !w || !part || !workspace) return CCDC_EINVAL;
     const ccdc_plan_s &P = *plan;
-    if (P.dtype != CCDC_F32) return CCDC_ESTATE;
+    if (P.dtype != CCDC_F32 || P.compression_mode) return CCDC_ESTATE;
     const long long d = P.row_elems;
     if (rows < 16 || rows % 16 != 0 || rows > 4096 || d % 512 != 0 || d > 65536) return CCDC_ESIZE;
     MapParams mp;
     std::memset(&mp, 0, sizeof(mp));
     for (int k = 0; k < P.K; ++k) {
-        mp.first_job[k + 1] = mp.first_job[k] + P.nlocal[k] * P.b;
+        mp.first_job[k + 1] = mp.first_job[k] + P.node_nfiles[k];
         if (P.nlocal[k] == 0) continue;
         if (!files_x[k] || !files_y[k] || !part[k]) return CCDC_EINVAL;
         if ((reinterpret_cast<uintptr_t>(files_x[k]) | reinterpret_cast<uintptr_t>(part[k])) & 15u) return CCDC_EINVAL;

@@ -98,6 +98,8 @@ int finish(ccdc_plan_s &P) {
             int k = P.batch_nodes[(size_t)p * r + i];
             P.slot[(size_t)k * P.nbatch + p] = P.nlocal[k]++;
         }
+    P.node_nfiles.assign(K, 0);
+    for (int k = 0; k < K; ++k) P.node_nfiles[k] = P.nlocal[k] * P.b;
     // who receives which batch in which round; every (batch, outside node) exactly once
     P.recv_round.assign((size_t)P.nbatch * K, -1);
     P.node_round_index.assign((size_t)P.nround * (r + 1), 0);
@@ -141,7 +143,7 @@ int finish(ccdc_plan_s &P) {
         for (int as = 0; as <= r; ++as) {
             const long long cr = g * (r + 1) + as;
             const int ks = S[as];
-            ccdc_row row{ks, 0, cr * P.s_pad, P.s, -1};
+            ccdc_row row{ks, 0, cr * P.s_pad, P.s, -1, 0};
             P.enc_fused.rows[cr] = row;
             P.enc_pk.rows[cr] = row;
             int n = 0;
@@ -163,7 +165,7 @@ int finish(ccdc_plan_s &P) {
             if (P.slot[(size_t)k * P.nbatch + p] < 0) continue;
             for (int t = 0; t < K; ++t) {
                 if (index_in(&P.batch_nodes[(size_t)p * r], r, t) >= 0) continue;
-                P.cmb.rows.push_back({k, k, packet_index(P, k, p, t) * P.len, P.len, -1});
+                P.cmb.rows.push_back({k, k, packet_index(P, k, p, t) * P.len, P.len, -1, 0});
                 P.cmb.refs.push_back({part_row(P, k, p, t), P.len});
             }
         }
@@ -182,7 +184,7 @@ int finish(ccdc_plan_s &P) {
                 const int i0 = index_in(&P.batch_nodes[(size_t)bat[ak] * r], r, ks);
                 const long long n0 = seg_valid(P, i0);
                 P.dec_pk.rows.push_back({k, k, n0 > 0 ? ridx * P.len + (long long)i0 * P.s : 0, n0,
-                                         (g * (r + 1) + as) * P.s_pad});
+                                         (g * (r + 1) + as) * P.s_pad, 0});
                 for (int a = 0; a <= r; ++a) {
                     if (a == ak || a == as) continue;
                     const int i = index_in(&P.batch_nodes[(size_t)bat[a] * r], r, ks);
@@ -385,9 +387,75 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
     }
 }
 
+// The appendix's compression-only scheme for one job, mu = r/K: m = ceil(K/r)
+// batches (the first m-1 of mu*N files, the last the rest), node k stores batch
+// k mod m, and for every batch t it lacks node k is sent one pre-combined packet
+// by the first node after k (cyclically) that stores batch t.
+int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
+    if (!out) return CCDC_EINVAL;
+    *out = nullptr;
+    int rc = check_parameters(K, r, N, Q, B, (int)dtype);
+    if (rc != CCDC_OK) return rc;
+    if (((long long)r * N) % K != 0) return CCDC_EINVAL;        // mu*N files per batch
+    const int m = (K + r - 1) / r;
+    const long long full = (long long)r * N / K, last = N - (long long)(m - 1) * full;
+    if (last < 1) return CCDC_EINVAL;
+    try {
+        ccdc_plan_s *pp = new ccdc_plan_s();
+        ccdc_plan_s &P = *pp;
+        P.K = K; P.r = r; P.N = N; P.Q = Q; P.B = B; P.dtype = (int)dtype; P.compression_mode = true;
+        P.J = 1; P.b = full; P.len = (long long)(Q / K) * B; P.s = P.len; P.s_pad = (P.s + 3) / 4 * 4;
+        P.row_elems = (long long)Q * B;
+        P.nbatch = m; P.nround = 0; P.nterm = m;
+        P.vec = P.len % 4 == 0 ? 4 : P.len % 2 == 0 ? 2 : 1;
+        P.term_stride = 2;
+        P.job_batch0.assign(1, 0);
+        P.batch_file0.resize(m); P.batch_job.assign(m, 0);
+        for (int t = 0; t < m; ++t) P.batch_file0[t] = t * full;
+        P.slot.assign((size_t)K * m, -1);
+        P.nlocal.assign(K, 1); P.node_nfiles.assign(K, 0); P.node_nrounds.assign(K, m - 1);
+        for (int k = 0; k < K; ++k) {
+            P.slot[(size_t)k * m + k % m] = 0;
+            P.node_nfiles[k] = (k % m == m - 1) ? last : full;
+        }
+        P.cmb.na = 1; P.cmb.n_max = P.len;
+        P.red_terms.resize((size_t)K * m);
+        for (int k = 0; k < K; ++k) {
+            int slot = 0;
+            for (int t = 0; t < m; ++t) {
+                const long long nf = t == m - 1 ? last : full;
+                if (t == k % m) {
+                    P.red_terms[(size_t)k * m + t] = {(long long)k * P.len, -nf};    // own batch, nf files
+                    continue;
+                }
+                int ks = (k + 1) % K;
+                while (ks % m != t) ks = (ks + 1) % K;
+                P.cmb.rows.push_back({ks, k, (long long)slot * P.len, P.len, -1, nf});
+                P.cmb.refs.push_back({(long long)k * P.len, P.len});
+                P.red_terms[(size_t)k * m + t] = {(long long)slot * P.len, 1};
+                ++slot;
+            }
+        }
+        *out = pp;
+        return CCDC_OK;
+    } catch (const std::bad_alloc &) {
+        return CCDC_ENOMEM;
+    }
+}
+
 }  // namespace
 
 extern "C" {
+
+int ccdc_plan_compression(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
+    return make_compression_plan(K, r, N, Q, B, dtype, out);
+}
+
+long long ccdc_plan_batch_files(const ccdc_plan_t *p, long long b) {
+    if (!p || b < 0 || b >= p->nbatch) return 0;
+    if (p->compression_mode && b == p->nbatch - 1) return p->N - (p->nbatch - 1) * p->b;
+    return p->b;
+}
 
 int ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
     return make_plan(K, r, N, Q, B, dtype, false, out);
@@ -410,10 +478,21 @@ long long ccdc_plan_files_per_batch(const ccdc_plan_t *p) { return p ? p->b : 0;
 long long ccdc_plan_packet_elems(const ccdc_plan_t *p) { return p ? p->len : 0; }
 long long ccdc_plan_segment_elems(const ccdc_plan_t *p) { return p ? p->s : 0; }
 long long ccdc_plan_coded_row_elems(const ccdc_plan_t *p) { return p ? p->s_pad : 0; }
-long long ccdc_plan_coded_bits(const ccdc_plan_t *p) { return p ? p->nround * (p->r + 1) * 32 * p->s : 0; }
+long long ccdc_plan_coded_bits(const ccdc_plan_t *p) {
+    if (!p) return 0;
+    if (p->compression_mode) return (long long)p->K * (p->nbatch - 1) * 32 * p->len;   // unicast packets
+    return p->nround * (p->r + 1) * 32 * p->s;
+}
 
 int ccdc_plan_batch_of_file(const ccdc_plan_t *p, long long n, int *nodes_out) {
     if (!p || !nodes_out || n < 0 || n >= p->J * p->N) return CCDC_EINVAL;
+    if (p->compression_mode) {      // holders of batch t: the nodes k with k mod m = t; padded with -1
+        const long long t = std::min<long long>(n / p->b, p->nbatch - 1);
+        int c = 0;
+        for (int k = 0; k < p->K && c < p->r; ++k) if (k % p->nbatch == t) nodes_out[c++] = k;
+        while (c < p->r) nodes_out[c++] = -1;
+        return CCDC_OK;
+    }
     const long long j = n / p->N, a = (n % p->N) / p->b;
     const long long b = p->job_batch0[j] + a;
     std::memcpy(nodes_out, &p->batch_nodes[(size_t)b * p->r], sizeof(int) * p->r);
@@ -422,6 +501,16 @@ int ccdc_plan_batch_of_file(const ccdc_plan_t *p, long long n, int *nodes_out) {
 
 int ccdc_plan_batch(const ccdc_plan_t *p, long long b, int *nodes_out, long long *first_file, long long *job) {
     if (!p || b < 0 || b >= p->nbatch) return CCDC_EINVAL;
+    if (p->compression_mode) {
+        if (nodes_out) {
+            int c = 0;
+            for (int k = 0; k < p->K && c < p->r; ++k) if (k % p->nbatch == b) nodes_out[c++] = k;
+            while (c < p->r) nodes_out[c++] = -1;
+        }
+        if (first_file) *first_file = p->batch_file0[b];
+        if (job) *job = 0;
+        return CCDC_OK;
+    }
     if (nodes_out) std::memcpy(nodes_out, &p->batch_nodes[(size_t)b * p->r], sizeof(int) * p->r);
     if (first_file) *first_file = p->batch_file0[b];
     if (job) *job = p->batch_job[b];
@@ -452,11 +541,12 @@ long long ccdc_plan_node_batches(const ccdc_plan_t *p, int k, long long *ids_out
 
 size_t ccdc_partition_bytes(const ccdc_plan_t *p, int k) {
     if (!p || k < 0 || k >= p->K) return 0;
-    return (size_t)(p->nlocal[k] * p->b * p->row_elems) * 4;
+    return (size_t)(p->node_nfiles[k] * p->row_elems) * 4;
 }
 
 size_t ccdc_packets_bytes(const ccdc_plan_t *p, int k) {
     if (!p || k < 0 || k >= p->K) return 0;
+    if (p->compression_mode) return 0;
     return (size_t)(p->nlocal[k] * (p->K - p->r) * p->len) * 4;
 }
 

@@ -6,6 +6,8 @@ fixed: files ascending, starting from the first file's value); outputs within
 1e-5 * sum_n |v_{q,n}| element-wise, the tolerance the method's evaluation
 states, since the fused path may add the per-batch terms in another grouping.
 """
+from math import comb
+
 import numpy as np
 import pytest
 
@@ -196,6 +198,38 @@ def test_special_float_patterns_survive_coding(ccdc):
                           o.coded().reshape(-1, plan.segment_elems))
     for k in range(K):
         assert np.array_equal(bits(decoded[k]).reshape(-1, B), o.decoded(k))
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", [(4, 2, 8, 4, 64), (6, 1, 12, 12, 33), (5, 2, 10, 5, 2 * 2048 + 12),
+                                       (8, 3, 16, 8, 1000), (5, 4, 10, 5, 7), (10, 2, 50, 10, 4096)])
+def test_compression_only_matches_oracle(ccdc, K, r, N, Q, B, dtype):
+    """The appendix's compression-only shuffle (comparator): every unicast packet and
+    every output bit-exact (same addition order on both sides), bits = ceil(1/mu)-1."""
+    from oracle.ccdc_oracle import compression_only
+
+    v = values_numpy(N, Q, B, dtype, seed=K + r)
+    ref_out, ref_recv, ref_bits, files = compression_only(K, r, N, Q, B, dtype, v)
+    plan = ccdc.Plan(K, r, N, Q, B, dtype, compression=True)
+    assert plan.coded_bits == ref_bits
+    assert [len(plan.node_files(k)) for k in range(K)] == files
+    part = plan.alloc_partitions()
+    plan.fill_partitions(part, torch.from_numpy(v).cuda())
+    recv = plan.alloc_decoded()
+    out_w, out = guarded(Q * B, plan.torch_dtype)
+    plan.compression_shuffle(part, recv, out)
+    torch.cuda.synchronize()
+    for k in range(K):
+        assert np.array_equal(bits(recv[k]).reshape(ref_recv.shape[1], -1), ref_recv[k])
+    assert np.array_equal(bits(out).reshape(Q, B), ref_out.view(np.uint32))
+    assert canaries_intact(out_w, Q * B)
+    # the coded steps refuse such a plan
+    with pytest.raises(ccdc.CcdcError) as e:
+        plan.encode_fused(part, out)
+    assert e.value.status == ccdc.ESTATE
+    with pytest.raises(ccdc.CcdcError) as e:
+        ccdc.Plan(K, r, comb(K, r) * 2, Q, B, dtype).compression_shuffle(part, recv, out)
+    assert e.value.status == ccdc.ESTATE
 
 
 def test_bad_arguments_are_refused(ccdc):

@@ -116,3 +116,29 @@ def test_storage_and_replication():
     assert sorted(seen) == list(range(N))
     assert all(len(v) == r and v == p.batch_of_file(n) for n, v in seen.items())
     assert [p.batch(b)[0] for b in range(p.num_batches)] == [list(c) for c in combinations(range(K), r)]
+
+
+@pytest.mark.parametrize("K,r,N", [(4, 2, 8), (6, 1, 12), (5, 2, 10), (8, 3, 16), (5, 4, 10), (20, 2, 190)])
+def test_compression_plan(K, r, N):
+    """Appendix placement: m = ceil(1/mu) batches, node k stores batch k mod m, at most
+    mu*N files per node; unicast bit count = (ceil(1/mu)-1) * Q * T."""
+    from fractions import Fraction
+
+    Q, B = K, 8
+    p = ccdc.Plan(K, r, N, Q, B, "float32", compression=True)
+    m = -(-K // r)
+    assert p.num_batches == m and p.num_groups == 0 and p.J == 1
+    assert Fraction(p.coded_bits, Q * 32 * B) == m - 1
+    seen = set()
+    for k in range(K):
+        files = p.node_files(k)
+        assert len(files) * K <= r * N and p.partition_bytes(k) == len(files) * Q * B * 4
+        assert p.node_batches(k) == [k % m]
+        assert p.decoded_bytes(k) == (m - 1) * (Q // K) * B * 4
+        for n in files:
+            assert k in p.batch_of_file(n)
+        seen.update(files)
+    assert seen == set(range(N))
+    assert p.coded_bytes == 0 and p.workspace_bytes == 0
+    with pytest.raises(ccdc.CcdcError):
+        ccdc.Plan(5, 2, 11, 5, 8, "float32", compression=True)      # mu*N not an integer
