@@ -157,8 +157,8 @@ def oracle_sample_shape(w, target_seconds):
     from oracle.ccdc_oracle import Oracle
 
     probe_B = w.r * 64
-    o = Oracle(w.K, w.r, w.N, w.Q, probe_B, w.dtype)
-    o.load_values(values_numpy(w.N, w.Q, probe_B, w.dtype, std=w.std))
+    o = Oracle(w.K, w.r, w.N, w.Q, probe_B, w.dtype, mode="paper" if w.jobs else "single")
+    o.load_values(values_numpy(o.J * w.N, w.Q, probe_B, w.dtype, std=w.std))
     t0 = time.perf_counter()
     o.shuffle(); o.reduce()
     per_elem = (time.perf_counter() - t0) / probe_B
@@ -171,11 +171,21 @@ def time_oracle(w, B):
     node memories is not part of the shuffle and is not timed)."""
     from oracle.ccdc_oracle import Oracle
 
-    o = Oracle(w.K, w.r, w.N, w.Q, B, w.dtype)
-    o.load_values(values_numpy(w.N, w.Q, B, w.dtype, std=w.std))
+    o = Oracle(w.K, w.r, w.N, w.Q, B, w.dtype, mode="paper" if w.jobs else "single")
+    o.load_values(values_numpy(o.J * w.N, w.Q, B, w.dtype, std=w.std))
     t0 = time.perf_counter()
     o.shuffle(); o.reduce()
     return time.perf_counter() - t0
+
+
+def sample_bytes(w, B):
+    """algorithmic bytes of the workload's structure at value length B."""
+    from math import comb
+
+    if w.jobs:
+        J = comb(w.K, w.r + 1)
+        return algorithmic_bytes(w.K, w.r, w.N, w.Q, B, J=J, rounds=J * (w.K - w.r))
+    return algorithmic_bytes(w.K, w.r, w.N, w.Q, B)
 
 
 def run_reference(args, w):
@@ -188,7 +198,7 @@ def run_reference(args, w):
         time_oracle(w, B)
     t = [time_oracle(w, B) for _ in range(args.steps)]
     per_step = sum(t) / len(t)
-    by = algorithmic_bytes(w.K, w.r, w.N, w.Q, B)
+    by = sample_bytes(w, B)
     value = by["iv_read"] / per_step / 1e9
     sample = f"{w.name} with B={B} of {w.B} elements per value (same K, r, N, Q), one pass per step"
     print(json.dumps({
@@ -230,13 +240,13 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
-    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=w.jobs)
     plan.upload()
     part = plan.alloc_partitions(dev)
     coded = plan.alloc(plan.coded_bytes, dev)
     out = plan.alloc(plan.out_bytes, dev)
     ws = plan.alloc(plan.workspace_bytes, dev)
-    by = algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B)
+    by = algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B, J=plan.J, rounds=plan.num_groups)
     stream = torch.cuda.current_stream()
     stages = []
     map_bytes = 0
@@ -258,7 +268,7 @@ def run_ours(args, w):
                        lambda: plan.map(files_x, files_y, wvec, w.map_rows, part, map_ws)))
     else:
         # every rank is an independent job of the same shape: its own seed
-        plan.fill_partitions_streaming(part, values_torch(w.N, w.Q, w.B, w.dtype, dev, seed=rank_seed(rank),
+        plan.fill_partitions_streaming(part, values_torch(plan.J * w.N, w.Q, w.B, w.dtype, dev, seed=rank_seed(rank),
                                                           std=w.std))
     stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
     stages.append(("k_decode_reduce", lambda: plan.decode_reduce(part, coded, out, ws)))
@@ -361,7 +371,7 @@ def run_ours(args, w):
     if world == 1 and not args.skip_cpu_baseline:
         Bs = oracle_sample_shape(w, 15.0)
         secs = time_oracle(w, Bs)
-        bs = algorithmic_bytes(w.K, w.r, w.N, w.Q, Bs)
+        bs = sample_bytes(w, Bs)
         cpu = {"value": bs["iv_read"] / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{w.name} with B={Bs} of {w.B} elements per value (same K, r, N, Q), one pass, "
                          f"{secs:.1f} s"}
@@ -373,7 +383,8 @@ def run_ours(args, w):
         "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
                    "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
                           f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written between steps, steps timed one by one"),
-                   "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": 1,
+                   "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": plan.J,
+                   "load_per_JQT": plan.coded_bits / (plan.J * w.Q * 32 * w.B),
                    "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
                    "algorithmic_bytes_per_step": by["total"] + map_bytes,
                    "hbm_frac_whole_step": (by["total"] + map_bytes) / (ms_per_step * 1e-3) / 1e9 / peak},

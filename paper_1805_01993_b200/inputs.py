@@ -20,6 +20,8 @@ The five named workloads are the shapes the method is evaluated on:
         gradient per file cut into 20 slices
   cfg5  K=8  r=3 N=112  Q=8  B=1024     fp32, produced by the linear-regression
         Map from files X_n (512 x 8192, bf16-representable), y_n, and w
+plus ``jobs20``: the paper's J = C(K, r+1) parallel jobs at K=20, r=2 (1140 jobs of 21
+files each, B=10240), sized like cfg4.
 """
 from __future__ import annotations
 
@@ -41,6 +43,7 @@ class Workload:
     dtype: str            # "int32" | "float32"
     std: float = 1.0      # standard deviation of the normal draws (fp32 only)
     map_rows: int = 0     # linear-regression workload: rows m of X_n (0 = no Map)
+    jobs: bool = False    # the scheme as stated for J = C(K, r+1) jobs (stages 1 and 2); N is per job
 
     @property
     def map_cols(self) -> int:
@@ -57,6 +60,9 @@ CONFIGS = {
     "cfg3": Workload("cfg3", 16, 4, 1820, 16, 16384, "float32"),
     "cfg4": Workload("cfg4", 20, 2, 190, 20, 1280000, "float32", std=float(np.sqrt(1e-3))),
     "cfg5": Workload("cfg5", 8, 3, 112, 8, 1024, "float32", map_rows=512),
+    # the paper's own multi-job setting at the scale of cfg4: J = C(20,3) = 1140 jobs of 21 files,
+    # 2394 files (1.96 GB) per node, load (1-mu)(mu K+1)/(mu K) = 1.35
+    "jobs20": Workload("jobs20", 20, 2, 21, 20, 10240, "float32", std=float(np.sqrt(1e-3)), jobs=True),
 }
 
 
