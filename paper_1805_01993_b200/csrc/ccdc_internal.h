@@ -18,6 +18,9 @@
 #ifndef CCDC_DECODE_VECTORS
 #define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
+#ifndef CCDC_DECODE_DEPTH
+#define CCDC_DECODE_DEPTH 2         // batches whose loads are issued together (one-file batches, r <= 4)
+#endif
 #ifndef CCDC_GATHER_THREADS
 #define CCDC_GATHER_THREADS 128
 #endif

@@ -265,7 +265,11 @@ struct DecodeParams {
     int stage_terms;        // terms staged in shared memory at a time
 };
 
-template <int VEC, bool F32, int NT>
+// R1S >= 0: the plan has one file per batch and r-1 = R1S; then the loads of
+// DEPTH consecutive batches are issued together before any is consumed (about
+// 64 KiB of loads in flight per SM is what the HBM read rate needs).
+// R1S < 0: any r and b, batch by batch.
+template <int VEC, bool F32, int NT, int R1S>
 __global__ void __launch_bounds__(NT)
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
     constexpr long long TILE = (long long)NT * VEC * DUNROLL;
@@ -298,35 +302,76 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
         __syncthreads();
         for (int x = threadIdx.x; x < nt * p.TS; x += NT) sh_terms[x] = table[t0 * p.TS + x];
         __syncthreads();
-        for (int t = 0; t < nt; ++t) {
-            const ccdc_ref *e = sh_terms + t * p.TS;
-            const long long coded_off = e[0].off;
-            Words<VEC> v[DUNROLL];
-            if (coded_off < 0) {
-                const ccdc_ref E = e[1];
+        if constexpr (R1S >= 0) {
+            constexpr int DEPTH = CCDC_DECODE_DEPTH;
+            for (int t = 0; t < nt; t += DEPTH) {
+                Words<VEC> v[DEPTH][1 + R1S][DUNROLL];
 #pragma unroll
-                for (int u = 0; u < DUNROLL; ++u) {
-                    const long long j = j0 + (long long)u * NT * VEC;
-                    v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
-                }
-            } else {
-#pragma unroll
-                for (int u = 0; u < DUNROLL; ++u) {
-                    const long long j = j0 + (long long)u * NT * VEC;
-                    v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
-                }
-                for (int c = 1; c <= r1; ++c) {
-                    const ccdc_ref E = e[c];
+                for (int x = 0; x < DEPTH; ++x) {              // every load of DEPTH batches first
+                    if (t + x >= nt) break;
+                    const ccdc_ref *e = sh_terms + (t + x) * p.TS;
+                    const long long coded_off = e[0].off;
 #pragma unroll
                     for (int u = 0; u < DUNROLL; ++u) {
                         const long long j = j0 + (long long)u * NT * VEC;
-                        if (j < seglen)
-                            xor_into<VEC>(v[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+                        if (coded_off < 0) {
+                            v[x][0][u] = j < seglen ? load_words<VEC>(src + e[1].off + j) : zero_words<VEC>();
+                        } else {
+                            v[x][0][u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
+#pragma unroll
+                            for (int c = 1; c <= R1S; ++c)
+                                v[x][c][u] = (j < seglen && j < e[c].vl) ? load_words<VEC>(src + e[c].off + j)
+                                                                         : zero_words<VEC>();
+                        }
+                    }
+                }
+#pragma unroll
+                for (int x = 0; x < DEPTH; ++x) {              // then consume them in batch order
+                    if (t + x >= nt) break;
+                    const bool local = sh_terms[(t + x) * p.TS].off < 0;
+#pragma unroll
+                    for (int u = 0; u < DUNROLL; ++u) {
+                        Words<VEC> val = v[x][0][u];
+                        if (!local) {
+#pragma unroll
+                            for (int c = 1; c <= R1S; ++c) xor_into<VEC>(val, v[x][c][u]);
+                        }
+                        add_into<VEC, F32>(acc[u], val);
                     }
                 }
             }
-#pragma unroll
-            for (int u = 0; u < DUNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
+        } else {
+            for (int t = 0; t < nt; ++t) {
+                const ccdc_ref *e = sh_terms + t * p.TS;
+                const long long coded_off = e[0].off;
+                Words<VEC> v[DUNROLL];
+                if (coded_off < 0) {
+                    const ccdc_ref E = e[1];
+    #pragma unroll
+                    for (int u = 0; u < DUNROLL; ++u) {
+                        const long long j = j0 + (long long)u * NT * VEC;
+                        v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
+                    }
+                } else {
+    #pragma unroll
+                    for (int u = 0; u < DUNROLL; ++u) {
+                        const long long j = j0 + (long long)u * NT * VEC;
+                        v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
+                    }
+                    for (int c = 1; c <= r1; ++c) {
+                        const ccdc_ref E = e[c];
+    #pragma unroll
+                        for (int u = 0; u < DUNROLL; ++u) {
+                            const long long j = j0 + (long long)u * NT * VEC;
+                            if (j < seglen)
+                                xor_into<VEC>(v[u], batch_sum<VEC, F32>(src, E.off, j, E.vl, p.b, p.file_stride));
+                        }
+                    }
+                }
+    #pragma unroll
+                for (int u = 0; u < DUNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
+            }
+    
         }
     }
     uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) +
@@ -627,10 +672,23 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
-        if (P.decode_threads == CCDC_DECODE_THREADS_SHORT)
-            k_decode_reduce<VEC, F32, CCDC_DECODE_THREADS_SHORT><<<(unsigned)blocks, CCDC_DECODE_THREADS_SHORT, smem, st>>>(dp);
-        else
-            k_decode_reduce<VEC, F32, DTHREADS><<<(unsigned)blocks, DTHREADS, smem, st>>>(dp);
+        // one file per batch and small r: the deep-load instantiation for that r
+        const int r1s = (P.b == 1 && P.r >= 2 && P.r <= 4) ? P.r - 1 : -1;
+        auto launch = [&](auto nt, auto r1) {
+            constexpr int NT = decltype(nt)::value;
+            constexpr int R1 = decltype(r1)::value;
+            k_decode_reduce<VEC, F32, NT, R1><<<(unsigned)blocks, NT, smem, st>>>(dp);
+        };
+        auto with_threads = [&](auto r1) {
+            if (P.decode_threads == CCDC_DECODE_THREADS_SHORT) launch(std::integral_constant<int, CCDC_DECODE_THREADS_SHORT>(), r1);
+            else launch(std::integral_constant<int, DTHREADS>(), r1);
+        };
+        switch (r1s) {
+        case 1: with_threads(std::integral_constant<int, 1>()); break;
+        case 2: with_threads(std::integral_constant<int, 2>()); break;
+        case 3: with_threads(std::integral_constant<int, 3>()); break;
+        default: with_threads(std::integral_constant<int, -1>()); break;
+        }
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
         const long long n = dp.nout * P.len;
