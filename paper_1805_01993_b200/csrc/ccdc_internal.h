@@ -58,6 +58,7 @@ struct ccdc_gather_table {
     std::vector<ccdc_ref> refs;     // [rows][na]
     int na = 0;
     long long n_max = 0;            // largest row length
+    bool uniform = true;            // no row carries its own file count (nf = 0 everywhere)
     // device copies
     const ccdc_row *d_rows = nullptr;
     const ccdc_ref *d_refs = nullptr;

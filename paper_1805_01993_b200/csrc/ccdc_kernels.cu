@@ -244,6 +244,54 @@ k_gather(const __grid_constant__ GatherParams p) {
     }
 }
 
+// Lean variant for the common shape of the fused encode: RS operands known at
+// compile time, one file per batch, no coded input.  All RS x SVEC loads of a
+// tile are issued from registers before the first XOR; no shared memory.
+#ifndef CCDC_STATIC_GATHER_THREADS
+#define CCDC_STATIC_GATHER_THREADS 256
+#endif
+#ifndef CCDC_STATIC_GATHER_VECTORS
+#define CCDC_STATIC_GATHER_VECTORS 2
+#endif
+constexpr int STHREADS = CCDC_STATIC_GATHER_THREADS;
+constexpr int SUNROLL = CCDC_STATIC_GATHER_VECTORS;
+
+template <int VEC, int RS>
+__global__ void __launch_bounds__(STHREADS)
+k_gather_static(const __grid_constant__ GatherParams p) {
+    constexpr long long TILE = (long long)STHREADS * VEC * SUNROLL;
+    const long long item = blockIdx.x;
+    const long long row = item / p.spans_per_row;
+    const long long span = item - row * p.spans_per_row;
+    if (row >= p.nrows) return;
+    const ccdc_row R = p.rows[row];
+    const long long begin = span * p.span_elems;
+    const long long end = min(R.n, begin + p.span_elems);
+    if (begin >= end) return;
+    ccdc_ref E[RS];
+#pragma unroll
+    for (int a = 0; a < RS; ++a) E[a] = p.refs[row * RS + a];
+    const uint32_t *src = p.src[R.src_node];
+    uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
+    for (long long base = begin; base < end; base += TILE) {
+        Words<VEC> v[RS][SUNROLL];
+#pragma unroll
+        for (int a = 0; a < RS; ++a)
+#pragma unroll
+            for (int u = 0; u < SUNROLL; ++u) {
+                const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+                v[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + j) : zero_words<VEC>();
+            }
+#pragma unroll
+        for (int u = 0; u < SUNROLL; ++u) {
+            const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+#pragma unroll
+            for (int a = 1; a < RS; ++a) xor_into<VEC>(v[0][u], v[a][u]);
+            if (j < end) store_words<VEC>(dst + j, v[0][u]);
+        }
+    }
+}
+
 // ------------------------------------------------------ fused decode + reduce
 // One block: node k (row of outputs), one segment i, one tile of it, one chunk
 // of the job's batches.  For each batch, ascending: the locally pre-combined
@@ -484,7 +532,8 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const long long tile = (long long)GTHREADS * VEC * GUNROLL;
+        const bool lean = b == 1 && !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
+        const long long tile = lean ? (long long)STHREADS * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 148 SMs x 16 blocks
         long long tiles = 32;
@@ -493,6 +542,16 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         gp.spans_per_row = (T.n_max + gp.span_elems - 1) / gp.span_elems;
         const long long blocks = gp.nrows * gp.spans_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
+        if (lean) {
+            // XOR of single files is the same for both dtypes: no addition happens
+            switch (T.na) {
+            case 1: k_gather_static<VEC, 1><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
+            case 2: k_gather_static<VEC, 2><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
+            case 3: k_gather_static<VEC, 3><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
+            default: k_gather_static<VEC, 4><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
+            }
+            return check_launch();
+        }
         const size_t smem = slots_bytes(VEC);
         int rc = allow_shared_memory(k_gather<VEC, F32>, smem);
         if (rc != CCDC_OK) return rc;

@@ -418,7 +418,7 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
             P.slot[(size_t)k * m + k % m] = 0;
             P.node_nfiles[k] = (k % m == m - 1) ? last : full;
         }
-        P.cmb.na = 1; P.cmb.n_max = P.len;
+        P.cmb.na = 1; P.cmb.n_max = P.len; P.cmb.uniform = false;
         P.red_terms.resize((size_t)K * m);
         for (int k = 0; k < K; ++k) {
             int slot = 0;

@@ -128,6 +128,11 @@ SHAPES = [
     (5, 3, 10, 5, 3 * 2049 + 1),            # vec 1, r does not divide B
     (6, 5, 12, 6, 7001),                    # r = K-1, one round
     (7, 3, 35, 14, 1000),                   # Q/K = 2
+    (32, 1, 32, 32, 40),                    # the largest K, r = 1
+    (32, 31, 32, 32, 70),                   # the largest K, r = K-1: one round of 32 members
+    (12, 6, 924, 12, 8),                    # 924 batches, 792 rounds of 7
+    (9, 5, 252, 9, 1030),                   # r = 5: general (run-time r) decode path, b = 2
+    (6, 2, 15, 6, 40000),                   # b = 1, long values: lean gather + deep-load decode
 ]
 
 

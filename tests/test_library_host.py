@@ -52,7 +52,7 @@ def test_invalid_parameters():
     assert ccdc.lib().ccdc_plan_num_groups(None) == 0
 
 
-SHAPES = [(3, 2, 6, 3, 8), (4, 2, 12, 4, 6), (4, 1, 8, 8, 3), (5, 3, 10, 10, 5), (5, 4, 5, 5, 2),
+SHAPES = [(32, 1, 32, 32, 4), (32, 31, 32, 32, 4), (12, 6, 924, 12, 2), (3, 2, 6, 3, 8), (4, 2, 12, 4, 6), (4, 1, 8, 8, 3), (5, 3, 10, 10, 5), (5, 4, 5, 5, 2),
           (6, 3, 40, 6, 4), (7, 2, 21, 7, 9), (10, 3, 480, 10, 16)]
 
 
