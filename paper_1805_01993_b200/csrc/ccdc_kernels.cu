@@ -244,9 +244,10 @@ k_gather(const __grid_constant__ GatherParams p) {
     }
 }
 
-// Lean variant for the common shape of the fused encode: RS operands known at
-// compile time, one file per batch, no coded input.  All RS x SVEC loads of a
-// tile are issued from registers before the first XOR; no shared memory.
+// Lean variant for the common shapes: RS operands known at compile time, no
+// coded input, every row summing the plan's b files.  The RS x SUNROLL loads
+// of a file step are issued from registers before they are consumed; no shared
+// memory, no barrier.
 #ifndef CCDC_STATIC_GATHER_THREADS
 #define CCDC_STATIC_GATHER_THREADS 256
 #endif
@@ -256,7 +257,7 @@ k_gather(const __grid_constant__ GatherParams p) {
 constexpr int STHREADS = CCDC_STATIC_GATHER_THREADS;
 constexpr int SUNROLL = CCDC_STATIC_GATHER_VECTORS;
 
-template <int VEC, int RS>
+template <int VEC, bool F32, int RS, bool B1>
 __global__ void __launch_bounds__(STHREADS)
 k_gather_static(const __grid_constant__ GatherParams p) {
     constexpr long long TILE = (long long)STHREADS * VEC * SUNROLL;
@@ -282,6 +283,21 @@ k_gather_static(const __grid_constant__ GatherParams p) {
                 const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
                 v[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + j) : zero_words<VEC>();
             }
+        for (int f = 1; !B1 && f < p.b; ++f) {      // the other files of each batch, ascending
+            Words<VEC> w[RS][SUNROLL];
+#pragma unroll
+            for (int a = 0; a < RS; ++a)
+#pragma unroll
+                for (int u = 0; u < SUNROLL; ++u) {
+                    const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+                    w[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + f * p.file_stride + j)
+                                                       : zero_words<VEC>();
+                }
+#pragma unroll
+            for (int a = 0; a < RS; ++a)
+#pragma unroll
+                for (int u = 0; u < SUNROLL; ++u) add_into<VEC, F32>(v[a][u], w[a][u]);
+        }
 #pragma unroll
         for (int u = 0; u < SUNROLL; ++u) {
             const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
@@ -313,11 +329,11 @@ struct DecodeParams {
     int stage_terms;        // terms staged in shared memory at a time
 };
 
-// R1S >= 0: the plan has one file per batch and r-1 = R1S; then the loads of
-// DEPTH consecutive batches are issued together before any is consumed (about
-// 64 KiB of loads in flight per SM is what the HBM read rate needs).
-// R1S < 0: any r and b, batch by batch.
-template <int VEC, bool F32, int NT, int R1S>
+// R1S >= 0: r-1 = R1S is a compile-time constant, so a batch's loads are issued
+// together; with one file per batch (B1) the loads of DEPTH consecutive batches
+// are issued before any is consumed (about 64 KiB of loads in flight per SM is
+// what the HBM read rate needs).  R1S < 0: any r, batch by batch.
+template <int VEC, bool F32, int NT, int R1S, bool B1>
 __global__ void __launch_bounds__(NT)
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
     constexpr long long TILE = (long long)NT * VEC * DUNROLL;
@@ -351,7 +367,12 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
         for (int x = threadIdx.x; x < nt * p.TS; x += NT) sh_terms[x] = table[t0 * p.TS + x];
         __syncthreads();
         if constexpr (R1S >= 0) {
-            constexpr int DEPTH = CCDC_DECODE_DEPTH;
+            constexpr int DEPTH = B1 ? CCDC_DECODE_DEPTH : 1;
+            // one operand: a single word vector, or the batch sum over its b files
+            auto fetch = [&](long long off, long long j, long long vl) -> Words<VEC> {
+                if (B1) return j < vl ? load_words<VEC>(src + off + j) : zero_words<VEC>();
+                return batch_sum<VEC, F32>(src, off, j, vl, p.b, p.file_stride);
+            };
             for (int t = 0; t < nt; t += DEPTH) {
                 Words<VEC> v[DEPTH][1 + R1S][DUNROLL];
 #pragma unroll
@@ -363,13 +384,12 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                     for (int u = 0; u < DUNROLL; ++u) {
                         const long long j = j0 + (long long)u * NT * VEC;
                         if (coded_off < 0) {
-                            v[x][0][u] = j < seglen ? load_words<VEC>(src + e[1].off + j) : zero_words<VEC>();
+                            v[x][0][u] = fetch(e[1].off, j, seglen);
                         } else {
                             v[x][0][u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
 #pragma unroll
                             for (int c = 1; c <= R1S; ++c)
-                                v[x][c][u] = (j < seglen && j < e[c].vl) ? load_words<VEC>(src + e[c].off + j)
-                                                                         : zero_words<VEC>();
+                                v[x][c][u] = fetch(e[c].off, j, min(seglen, e[c].vl));
                         }
                     }
                 }
@@ -532,7 +552,7 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const bool lean = b == 1 && !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
+        const bool lean = !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
         const long long tile = lean ? (long long)STHREADS * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 148 SMs x 16 blocks
@@ -543,12 +563,16 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         const long long blocks = gp.nrows * gp.spans_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         if (lean) {
-            // XOR of single files is the same for both dtypes: no addition happens
+            auto go = [&](auto rs) {
+                constexpr int RS = decltype(rs)::value;
+                if (b == 1) k_gather_static<VEC, F32, RS, true><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
+                else k_gather_static<VEC, F32, RS, false><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
+            };
             switch (T.na) {
-            case 1: k_gather_static<VEC, 1><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
-            case 2: k_gather_static<VEC, 2><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
-            case 3: k_gather_static<VEC, 3><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
-            default: k_gather_static<VEC, 4><<<(unsigned)blocks, STHREADS, 0, st>>>(gp); break;
+            case 1: go(std::integral_constant<int, 1>()); break;
+            case 2: go(std::integral_constant<int, 2>()); break;
+            case 3: go(std::integral_constant<int, 3>()); break;
+            default: go(std::integral_constant<int, 4>()); break;
             }
             return check_launch();
         }
@@ -731,22 +755,29 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
-        // one file per batch and small r: the deep-load instantiation for that r
-        const int r1s = (P.b == 1 && P.r >= 2 && P.r <= 4) ? P.r - 1 : -1;
-        auto launch = [&](auto nt, auto r1) {
+        // small r: the instantiation with r-1 as a compile-time constant
+        const int r1s = P.r <= 4 ? P.r - 1 : -1;
+        auto launch = [&](auto nt, auto r1, auto b1) {
             constexpr int NT = decltype(nt)::value;
             constexpr int R1 = decltype(r1)::value;
-            k_decode_reduce<VEC, F32, NT, R1><<<(unsigned)blocks, NT, smem, st>>>(dp);
+            constexpr bool B1 = decltype(b1)::value;
+            k_decode_reduce<VEC, F32, NT, R1, B1><<<(unsigned)blocks, NT, smem, st>>>(dp);
         };
-        auto with_threads = [&](auto r1) {
-            if (P.decode_threads == CCDC_DECODE_THREADS_SHORT) launch(std::integral_constant<int, CCDC_DECODE_THREADS_SHORT>(), r1);
-            else launch(std::integral_constant<int, DTHREADS>(), r1);
+        auto with_threads = [&](auto r1, auto b1) {
+            if (P.decode_threads == CCDC_DECODE_THREADS_SHORT) launch(std::integral_constant<int, CCDC_DECODE_THREADS_SHORT>(), r1, b1);
+            else launch(std::integral_constant<int, DTHREADS>(), r1, b1);
+        };
+        // several files per batch: the batch-by-batch path measured faster (J-job workload, b = 7)
+        auto with_files = [&](auto r1) {
+            if (P.b == 1) with_threads(r1, std::true_type());
+            else with_threads(std::integral_constant<int, -1>(), std::false_type());
         };
         switch (r1s) {
-        case 1: with_threads(std::integral_constant<int, 1>()); break;
-        case 2: with_threads(std::integral_constant<int, 2>()); break;
-        case 3: with_threads(std::integral_constant<int, 3>()); break;
-        default: with_threads(std::integral_constant<int, -1>()); break;
+        case 0: with_files(std::integral_constant<int, 0>()); break;
+        case 1: with_files(std::integral_constant<int, 1>()); break;
+        case 2: with_files(std::integral_constant<int, 2>()); break;
+        case 3: with_files(std::integral_constant<int, 3>()); break;
+        default: with_threads(std::integral_constant<int, -1>(), std::false_type()); break;
         }
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
