@@ -166,13 +166,18 @@ def oracle_sample_shape(w, target_seconds):
     return max(4 * w.r, min(B, w.B))
 
 
-def time_oracle(w, B):
-    """One oracle pass (shuffle + reduce; the copy of the Map outputs into the
-    node memories is not part of the shuffle and is not timed)."""
+def make_oracle(w, B):
+    """The oracle on the workload's structure at value length B, Map outputs placed."""
     from oracle.ccdc_oracle import Oracle
 
     o = Oracle(w.K, w.r, w.N, w.Q, B, w.dtype, mode="paper" if w.jobs else "single")
     o.load_values(values_numpy(o.J * w.N, w.Q, B, w.dtype, std=w.std))
+    return o
+
+
+def time_oracle(o):
+    """One oracle pass (shuffle + reduce; the copy of the Map outputs into the
+    node memories is not part of the shuffle and is not timed)."""
     t0 = time.perf_counter()
     o.shuffle(); o.reduce()
     return time.perf_counter() - t0
@@ -194,9 +199,10 @@ def run_reference(args, w):
         return
     total_budget = 150.0
     B = oracle_sample_shape(w, total_budget / (args.steps + args.warmup))
+    o = make_oracle(w, B)
     for _ in range(args.warmup):
-        time_oracle(w, B)
-    t = [time_oracle(w, B) for _ in range(args.steps)]
+        time_oracle(o)
+    t = [time_oracle(o) for _ in range(args.steps)]
     per_step = sum(t) / len(t)
     by = sample_bytes(w, B)
     value = by["iv_read"] / per_step / 1e9
@@ -370,7 +376,7 @@ def run_ours(args, w):
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
         Bs = oracle_sample_shape(w, 15.0)
-        secs = time_oracle(w, Bs)
+        secs = time_oracle(make_oracle(w, Bs))
         bs = sample_bytes(w, Bs)
         cpu = {"value": bs["iv_read"] / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{w.name} with B={Bs} of {w.B} elements per value (same K, r, N, Q), one pass, "
