@@ -30,7 +30,7 @@ namespace {
 #define CCDC_MAP_MIN_BLOCKS 2        // register budget: 65536 / (256 * MIN_BLOCKS) per thread
 #endif
 #ifndef CCDC_MAP_DEPTH1
-#define CCDC_MAP_DEPTH1 8            // pass 1: 32-column quarters per trip (2 loads each)
+#define CCDC_MAP_DEPTH1 8            // pass 1: 64-column steps per trip (2 loads each)
 #endif
 #ifndef CCDC_MAP_DEPTH2
 #define CCDC_MAP_DEPTH2 2            // pass 2: 16-row steps per trip (4 loads each)
@@ -93,13 +93,15 @@ __device__ __forceinline__ int node_of_job(const MapParams &p, long long job) {
 }
 
 // ---- pass 1: u = X w - y for 16 rows of one file.
-// The k index of the MMA is a free relabelling of the columns: thread (g, t)
-// of a warp loads 8 consecutive columns of rows g and g+8 with one 16-byte load
-// each and feeds them as k = 2t, 2t+1, 2t+8, 2t+9 of two MMAs; w is placed in
-// column n = 0 of B with the same relabelling (lanes with g = 0), the other
-// columns are zero.  The 8 warps split the columns; their partial dots are
-// added in warp order.
-template <int QUARTERS>     // 32-column quarters per loop trip: 2 * QUARTERS loads in flight per thread
+// Both the k index and the row index of the MMA are free relabellings.  A warp
+// step covers 8 rows x 64 columns with two fully coalesced loads (each 4 rows x
+// 128 bytes): thread (g, t) reads 16 bytes of row g/2 (and of row 4 + g/2) at
+// column 32 (g%2) + 8 t.  MMA row m = g thus holds half (g%2) of row g/2, so w
+// is placed in TWO columns of B: n = 0 the first 32 columns of the step, n = 1
+// the second 32 (lanes with g = 0, 1), and D[m][m%2] is that half's dot
+// product.  The 8 warps are 2 row groups x 4 column quarters; partial dots are
+// added in a fixed order.
+template <int QUARTERS>     // 64-column steps per loop trip: 2 * QUARTERS loads in flight per thread
 __device__ __forceinline__ void residual_block(const MapParams &p, const uint32_t *sh_w, float (*sh_part)[16],
                                                long long job, long long row0) {
     const int k = node_of_job(p, job);
@@ -107,37 +109,42 @@ __device__ __forceinline__ void residual_block(const MapParams &p, const uint32_
     const uint16_t *X = p.x[k] + (file * p.rows + row0) * p.d;
     const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
     const int g = lane / 4, t = lane % 4;
-    const long long cols_per_warp = p.d / MAP_WARPS;        // a multiple of 64
-    const uint16_t *rowA = X + (long long)g * p.d;
-    const uint16_t *rowB = X + (long long)(g + 8) * p.d;
+    const int row_group = warp & 1, quarter = warp >> 1;
+    const long long cols_per_warp = p.d / 4;                // a multiple of 64
+    const long long col_off = 32 * (g & 1) + 8 * t;
+    const uint16_t *rowA = X + (long long)(row_group * 8 + g / 2) * p.d + col_off;
+    const uint16_t *rowB = rowA + 4 * p.d;
     const uint64_t keep = l2_policy_keep();
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    for (long long c0 = warp * cols_per_warp; c0 < (warp + 1) * cols_per_warp; c0 += 32 * QUARTERS) {
+    for (long long c0 = quarter * cols_per_warp; c0 < (quarter + 1) * cols_per_warp; c0 += 64 * QUARTERS) {
         uint4 va[QUARTERS], vb[QUARTERS];
 #pragma unroll
         for (int q = 0; q < QUARTERS; ++q) {         // all loads of the trip first
-            const long long c = c0 + 32 * q + 8 * t;
-            va[q] = load_keep(rowA + c, keep);
-            vb[q] = load_keep(rowB + c, keep);
+            va[q] = load_keep(rowA + c0 + 64 * q, keep);
+            vb[q] = load_keep(rowB + c0 + 64 * q, keep);
         }
 #pragma unroll
         for (int q = 0; q < QUARTERS; ++q) {
-            const long long c = c0 + 32 * q + 8 * t;
             uint4 wv = make_uint4(0u, 0u, 0u, 0u);
-            if (g == 0) wv = *reinterpret_cast<const uint4 *>(sh_w + c / 2);
+            if (g < 2) wv = *reinterpret_cast<const uint4 *>(sh_w + (c0 + 64 * q + 32 * g + 8 * t) / 2);
             mma_bf16(acc, va[q].x, vb[q].x, va[q].y, vb[q].y, wv.x, wv.y);
             mma_bf16(acc, va[q].z, vb[q].z, va[q].w, vb[q].w, wv.z, wv.w);
         }
     }
-    // column n = 0 of the accumulator tile: thread (g, t = 0) holds rows g and g+8
+    // D[m][m%2]: lane (g, t = 0) holds columns 0, 1 of MMA rows g and g+8
     if (t == 0) {
-        sh_part[warp][g] = acc[0];
-        sh_part[warp][g + 8] = acc[2];
+        sh_part[warp][g] = (g & 1) ? acc[1] : acc[0];
+        sh_part[warp][g + 8] = (g & 1) ? acc[3] : acc[2];
     }
     __syncthreads();
     if (threadIdx.x < 16) {
-        float s = sh_part[0][threadIdx.x];
-        for (int wv = 1; wv < MAP_WARPS; ++wv) s += sh_part[wv][threadIdx.x];   // fixed order
+        const int rg = threadIdx.x / 8, rr = threadIdx.x % 8;           // row group, row inside it
+        const int m0 = rr < 4 ? 2 * rr : 8 + 2 * (rr - 4);              // its two half-rows in the MMA tile
+        float s = 0.f;
+        for (int qt = 0; qt < 4; ++qt) {                                // fixed order
+            const int wsrc = qt * 2 + rg;
+            s += sh_part[wsrc][m0] + sh_part[wsrc][m0 + 1];
+        }
         const long long r = row0 + threadIdx.x;
         p.u[job * p.rows + r] = s - p.y[k][file * p.rows + r];
         __threadfence();                    // the residuals are visible before the job's counter moves
@@ -269,7 +276,7 @@ k_map(const __grid_constant__ MapParams p) {
     const long long n1 = p.rows / 16, n2 = (p.d + GRAD_COLS - 1) / GRAD_COLS, per = n1 + n2;
     const long long total = (p.njobs + CCDC_MAP_LAG) * per;
     // deeper load pipelines when the shape divides evenly
-    const bool deep1 = (p.d / MAP_WARPS) % (32 * CCDC_MAP_DEPTH1) == 0;
+    const bool deep1 = (p.d / 4) % (64 * CCDC_MAP_DEPTH1) == 0;
     const bool deep2 = p.rows % (16 * CCDC_MAP_DEPTH2) == 0;
     for (;;) {
         __syncthreads();                        // sh_ticket, sh_u and sh_part are free again
@@ -281,7 +288,7 @@ k_map(const __grid_constant__ MapParams p) {
         if (slot < n1) {
             if (step < p.njobs) {
                 if (deep1) residual_block<CCDC_MAP_DEPTH1>(p, sh_w, sh_part, step, slot * 16);
-                else residual_block<2>(p, sh_w, sh_part, step, slot * 16);
+                else residual_block<1>(p, sh_w, sh_part, step, slot * 16);
             }
         } else {
             const long long job = step - CCDC_MAP_LAG;
