@@ -39,7 +39,7 @@ UNIT = "GB/s"
 # taken on the cfg4 structure with B = 128000; it grows in proportion to B.  Only
 # valid for the kernel sources it was measured on (hash below); otherwise null.
 NCU_TRAFFIC = {
-    "sources_sha256": "90c1652775e8a6181689fdd5443d19b8222297976ac13718ea4667c23ed40c62",
+    "sources_sha256": "9175ad87480a0119948c1248528a3e0a00dffa152e2847b9321208f2c83aa194",
     "workload": "cfg4", "value_elems": 128000, "decode_kernel_bytes": 3528858368.0 + 11559936.0,
 }
 

@@ -27,6 +27,9 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
  *     All step functions are asynchronous on it; a step that follows another
  *     on the same stream sees its results.
+ *   - A plan may be used by one host thread at a time and on one device: the
+ *     device that was current when its tables were uploaded (another device
+ *     gives CCDC_ESTATE).  Different plans are independent.
  *   - Elements are 32 bits wide: int32 with wrapping addition or IEEE binary32.
  *     XOR coding acts on the raw bit patterns in both cases.
  *

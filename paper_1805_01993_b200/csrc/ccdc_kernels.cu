@@ -5,6 +5,19 @@
 // loads in flight per thread, and tables of element offsets prepared by the
 // host planner.  A thread block that works for node k reads node k's buffers
 // and the shared coded buffer only.
+//
+//   k_gather_static   a destination row = XOR over a compile-time number of
+//                     operands of the batch sums of a segment (the fused encode,
+//                     the stepwise combine and encode); loads in registers
+//   k_gather          the same for any operand count, per-row file counts and
+//                     a coded input row (stepwise decode, compression-only
+//                     unicast); cp.async pipeline through shared memory
+//   k_decode_reduce   decode + cancel + reduce, decoded packets never stored
+//   k_sum_chunks      ordered sum of the partial outputs when the batch loop
+//                     of k_decode_reduce is split over blocks
+//   k_reduce          Eq. (1) from materialised packets (stepwise API)
+// No kernel waits on another block or thread: the encode -> decode dependency
+// is the boundary between two launches on one stream.
 #include <cuda_runtime.h>
 
 #include <atomic>
