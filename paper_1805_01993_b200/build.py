@@ -13,13 +13,14 @@ LIB = PKG / "libccdc.so"
 SOURCES = ["ccdc_plan.cpp", "ccdc_kernels.cu", "ccdc_map.cu"]
 
 
-def nvcc_command(out: Path, verbose: bool = False) -> list[str]:
+def nvcc_command(out: Path, verbose: bool = False, defines: tuple[str, ...] = ()) -> list[str]:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC,-Wall", "-shared", "-cudart", "static",
            "-I", str(ROOT / "include"), "-I", str(CSRC), "-o", str(out)]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += [f"-D{d}" for d in defines]
     return cmd + [str(CSRC / s) for s in SOURCES]
 
 
@@ -44,6 +45,14 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     os.replace(tmp, LIB)
     return LIB
+
+
+def build_variant(out: Path, defines: tuple[str, ...]) -> Path:
+    """Compile the library with extra -D options (build-time kernel choices) into ``out``."""
+    res = subprocess.run(nvcc_command(out, defines=defines), capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    return out
 
 
 if __name__ == "__main__":
