@@ -246,7 +246,12 @@ def run_ours(args, w):
             dist.barrier()
         torch.cuda.synchronize()
 
-    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=w.jobs)
+    # --shard-nodes: ONE job over all GPUs, K/N logical nodes per GPU, coded rows exchanged by an
+    # all-gather between the two launches (strong scaling).  Default: one independent job per GPU.
+    sharded = bool(args.shard_nodes) and world > 1
+    if sharded and (w.map_rows or w.K % world):
+        raise RuntimeError("--shard-nodes needs a shuffle-only workload and a GPU count that divides K")
+    plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=w.jobs, shard=(rank, world) if sharded else None)
     plan.upload()
     part = plan.alloc_partitions(dev)
     coded = plan.alloc(plan.coded_bytes, dev)
@@ -276,10 +281,17 @@ def run_ours(args, w):
         # every rank is an independent job of the same shape: its own seed
         plan.fill_partitions_streaming(part, values_torch(plan.J * w.N, w.Q, w.B, w.dtype, dev, seed=rank_seed(rank),
                                                           std=w.std))
-    stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
+    if sharded:
+        send = plan.alloc(plan.coded_send_bytes, dev)
+        stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, send)))
+        stages.append(("all_gather(coded rows)", lambda: dist.all_gather_into_tensor(coded, send)))
+    else:
+        stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
     stages.append(("k_decode_reduce", lambda: plan.decode_reduce(part, coded, out, ws)))
-    stage_bytes = {"k_map_residual+k_map_gradient": map_bytes, "k_gather(encode)": by["encode_kernel"],
-                   "k_decode_reduce": by["decode_kernel"]}
+    share = world if sharded else 1                      # a rank's part of the job
+    stage_bytes = {"k_map_residual+k_map_gradient": map_bytes, "k_gather(encode)": by["encode_kernel"] // share,
+                   "k_decode_reduce": by["decode_kernel"] // share,
+                   "all_gather(coded rows)": by["coded_write"] * (world - 1) // max(world, 1)}
     input_bytes = sum(plan.partition_bytes(k) for k in range(w.K)) + map_bytes
     # inputs that fit in L2 (126 MB) would be served from it on every repeat: flush between steps
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if input_bytes < (1 << 30) else None
@@ -318,15 +330,15 @@ def run_ours(args, w):
     stage_ms = {name: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
     enc_ms, dec_ms = stage_ms["k_gather(encode)"], stage_ms["k_decode_reduce"]
     ms_per_step = max_over_ranks(elapsed_ms, world, dev) / args.steps
-    value = whole_job_value(world, by["iv_read"], ms_per_step)
+    value = whole_job_value(1 if sharded else world, by["iv_read"], ms_per_step)
 
     # ---- end to end through the host-buffer entry point ------------------
     e2e = None
     try:
         if args.skip_e2e:
             raise RuntimeError("--skip-e2e")
-        if w.map_rows:
-            raise RuntimeError("host-buffer leg is defined for the shuffle-only workloads")
+        if w.map_rows or sharded:
+            raise RuntimeError("host-buffer leg is defined for the one-GPU shuffle-only workloads")
         import psutil
 
         need = sum(plan.partition_bytes(k) for k in range(w.K)) + plan.out_bytes
@@ -366,7 +378,8 @@ def run_ours(args, w):
         peak, peak_kind = json.loads(peaks_file.read_text())["hbm_gbs"], "measured"
     else:
         peak, peak_kind = 6650.0, "fallback"
-    top = max(stage_ms, key=stage_ms.get)                 # the dominant kernel of the step
+    # the dominant kernel of the step (the exchange between GPUs is reported beside it, not as a kernel)
+    top = max((n for n in stage_ms if not n.startswith("all_gather")), key=stage_ms.get)
     achieved = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
     others = {n: {"achieved": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9,
                   "frac": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / peak, "ms_per_launch": stage_ms[n]}
@@ -384,9 +397,11 @@ def run_ours(args, w):
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "strong" if sharded else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
+        "config": {"workload": w.name, "parallelism": f"nodes sharded over {world} GPUs, all-gather of coded rows" if sharded
+                   else f"{world} independent job(s), one per GPU", "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
                    "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
                           f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written between steps, steps timed one by one"),
                    "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": plan.J,
@@ -476,6 +491,8 @@ def main():
                     help="shorten every value to this many elements (profiling captures on a small case)")
     ap.add_argument("--scheme", choices=["ccdc", "compression"], default="ccdc",
                     help="compression = the appendix's compression-only shuffle, as a comparator")
+    ap.add_argument("--shard-nodes", action="store_true",
+                    help="with N > 1 GPUs: one job, K/N logical nodes per GPU, coded rows all-gathered (strong scaling)")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave out the oracle timing leg")
     args = ap.parse_args()

@@ -109,6 +109,27 @@ int  ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t 
  * Queries: ccdc_plan_num_batches = m, ccdc_plan_num_groups = 0, holders of a
  * batch are reported in r slots padded with -1. */
 int  ccdc_plan_compression(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
+/* ccdc_plan_sharded: the plan of ccdc_plan (jobs = 0) or ccdc_plan_jobs (jobs != 0)
+ * restricted to the logical nodes of one GPU out of `world` (the broadcast
+ * network of Section III becomes an all-gather between GPUs).  Requires
+ * world | K; node k lives on rank k / (K/world).  On such a plan
+ *   - pointer arrays still have K entries; only this rank's nodes are used;
+ *   - ccdc_encode_fused writes only the coded rows this rank's nodes send, packed
+ *     into a send buffer of ccdc_coded_send_bytes (the same on every rank);
+ *   - the caller gathers the send buffers of all ranks, rank-major, into a buffer
+ *     of ccdc_coded_bytes (e.g. ncclAllGather / all_gather_into_tensor): coded row
+ *     (round g, sender rank a) is then row ccdc_plan_coded_row_position(plan, g, a);
+ *   - ccdc_decode_reduce reads that gathered buffer and writes only the outputs of
+ *     this rank's nodes (out keeps its full [job][q][B] layout);
+ *   - ccdc_map maps only this rank's files; ccdc_shuffle and the stepwise calls
+ *     return CCDC_ESTATE.
+ * The bytes that cross between GPUs are the multicast bits of the scheme:
+ * ccdc_plan_coded_bits / 8 in total, each rank contributing 1/world. */
+int  ccdc_plan_sharded(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, int jobs, int rank,
+                       int world, ccdc_plan_t **out);
+long long ccdc_plan_coded_row_position(const ccdc_plan_t *plan, long long g, int a);
+int  ccdc_plan_node_is_local(const ccdc_plan_t *plan, int k);
+size_t ccdc_coded_send_bytes(const ccdc_plan_t *plan);
 void ccdc_plan_destroy(ccdc_plan_t *plan);
 
 /* Copies the schedule tables to the current device (cudaMalloc + cudaMemcpy,

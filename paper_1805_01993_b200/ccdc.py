@@ -28,6 +28,10 @@ SIGNATURES = {
     "ccdc_plan": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_jobs": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_compression": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
+    "ccdc_plan_sharded": (_I, [_I, _I, _LL, _I, _LL, _I, _I, _I, _I, _PP]),
+    "ccdc_plan_coded_row_position": (_LL, [_P, _LL, _I]),
+    "ccdc_plan_node_is_local": (_I, [_P, _I]),
+    "ccdc_coded_send_bytes": (_SZ, [_P]),
     "ccdc_plan_destroy": (None, [_P]),
     "ccdc_plan_upload": (_I, [_P]),
     "ccdc_plan_num_jobs": (_LL, [_P]),
@@ -115,14 +119,19 @@ def _stream_handle(stream):
 class Plan:
     """``ccdc_plan`` / ``ccdc_plan_jobs`` plus the step calls on torch tensors."""
 
-    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False, compression: bool = False):
+    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False, compression: bool = False, shard=None):
         self.K, self.r, self.N, self.Q, self.B = K, r, N, Q, B
         self.dtype = {"int32": I32, "float32": F32, I32: I32, F32: F32}[dtype]
         self.jobs = jobs
         h = ctypes.c_void_p()
         fn = lib().ccdc_plan_compression if compression else lib().ccdc_plan_jobs if jobs else lib().ccdc_plan
         self._h = None
-        _check(fn(K, r, N, Q, B, self.dtype, ctypes.byref(h)), "ccdc_plan")
+        self.shard = shard
+        if shard is not None:           # (rank, world): this GPU's share of the logical nodes
+            _check(lib().ccdc_plan_sharded(K, r, N, Q, B, self.dtype, int(jobs), shard[0], shard[1], ctypes.byref(h)),
+                   "ccdc_plan_sharded")
+        else:
+            _check(fn(K, r, N, Q, B, self.dtype, ctypes.byref(h)), "ccdc_plan")
         self._h = h
         L = lib()
         self.J = L.ccdc_plan_num_jobs(h)
@@ -176,6 +185,16 @@ class Plan:
     def decoded_bytes(self, k):
         return lib().ccdc_decoded_bytes(self._h, k)
 
+    def node_is_local(self, k):
+        return bool(lib().ccdc_plan_node_is_local(self._h, k))
+
+    def coded_row_position(self, g, a):
+        return lib().ccdc_plan_coded_row_position(self._h, g, a)
+
+    @property
+    def coded_send_bytes(self):
+        return lib().ccdc_coded_send_bytes(self._h)
+
     @property
     def coded_bytes(self):
         return lib().ccdc_coded_bytes(self._h)
@@ -212,7 +231,8 @@ class Plan:
         return torch.empty(max(nbytes // 4, 0), dtype=self.torch_dtype, device=device)
 
     def alloc_partitions(self, device="cuda"):
-        return [self.alloc(self.partition_bytes(k), device) for k in range(self.K)]
+        """one buffer per node (empty for nodes that live on another GPU)."""
+        return [self.alloc(self.partition_bytes(k) if self.node_is_local(k) else 0, device) for k in range(self.K)]
 
     def alloc_packets(self, device="cuda"):
         return [self.alloc(self.packets_bytes(k), device) for k in range(self.K)]
@@ -228,6 +248,8 @@ class Plan:
         row = self.Q * self.B
         flat = values.reshape(-1, row)
         for k in range(self.K):
+            if not self.node_is_local(k):
+                continue
             idx = torch.as_tensor(self.node_files(k), dtype=torch.long, device=flat.device)
             if idx.numel():
                 part[k].view(-1, row).copy_(flat.index_select(0, idx), non_blocking=False)
@@ -246,6 +268,8 @@ class Plan:
             sampled = torch.empty((self.J * self.N, self.Q, sample_index.numel()), dtype=self.torch_dtype)
         for n, t in file_iter:
             for k in self.batch_of_file(n):
+                if not self.node_is_local(k):
+                    continue
                 i = where[k][n]
                 part[k][i * row:(i + 1) * row].copy_(t.reshape(-1))
             if sampled is not None:

@@ -69,6 +69,12 @@ struct ccdc_plan_s {
     bool jobs_mode = false;
     bool compression_mode = false;  // the appendix's compression-only comparator (no coding)
     std::vector<long long> node_nfiles;     // [K] files stored at node k
+    // node-sharded plans (several GPUs, K/world nodes each): this rank's share
+    int shard_rank = 0, shard_world = 1;
+    long long send_rows = 0;                // coded rows this rank encodes (= every rank's)
+    std::vector<long long> coded_row_pos;   // [nround*(r+1)] position of a coded row in the gathered buffer
+    std::vector<int> out_rows;              // out rows (job*K + node) of this rank's nodes, ascending
+    const int *d_out_rows = nullptr;
     long long N = 0, B = 0, J = 1;
     long long b = 0;          // files per batch
     long long len = 0;        // (Q/K)*B

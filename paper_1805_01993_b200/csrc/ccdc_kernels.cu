@@ -333,6 +333,8 @@ struct DecodeParams {
     uint32_t *out;          // [out rows][len] when nchunk == 1
     uint32_t *ws;           // [nchunk][out rows][len] otherwise
     const ccdc_ref *terms;  // [out rows][r][nterm][TS]
+    const int *out_rows;    // the out rows to compute (node-sharded plans), or NULL for all
+    long long nlist;        // how many
     long long nout;         // out rows = J*K
     long long len, s;
     long long file_stride;
@@ -356,8 +358,9 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
     const long long tile = item % p.tiles_per_seg; item /= p.tiles_per_seg;
     const int i = (int)(item % p.r); item /= p.r;
     const int chunk = (int)(item % p.nchunk);
-    const long long orow = item / p.nchunk;
-    if (orow >= p.nout) return;
+    const long long li = item / p.nchunk;
+    if (li >= p.nlist) return;
+    const long long orow = p.out_rows ? p.out_rows[li] : li;
 
     const long long seglen = min(p.s, max(0LL, p.len - (long long)i * p.s));
     if (tile * TILE >= seglen) return;
@@ -467,9 +470,12 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
 // final pass of the split batch loop: out = ((ws[0] + ws[1]) + ...) in chunk order
 template <bool F32>
 __global__ void __launch_bounds__(DTHREADS)
-k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, long long n, int nchunk) {
-    const long long e = (long long)blockIdx.x * DTHREADS + threadIdx.x;
-    if (e >= n) return;
+k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, const int *__restrict__ out_rows,
+             long long nlist, long long len, long long n, int nchunk) {
+    const long long x = (long long)blockIdx.x * DTHREADS + threadIdx.x;
+    if (x >= nlist * len) return;
+    const long long li = x / len;
+    const long long e = (out_rows ? out_rows[li] : li) * len + (x - li * len);
     uint32_t acc = ws[e];
     for (int c = 1; c < nchunk; ++c) acc = add_word<F32>(acc, ws[(long long)c * n + e]);
     out[e] = acc;
@@ -546,8 +552,9 @@ int check_ptr_array(const ccdc_plan_s &P, const void *const *a, bool (*nonempty)
     return CCDC_OK;
 }
 
-bool has_part(const ccdc_plan_s &P, int k) { return P.nlocal[k] > 0; }
-bool has_decoded(const ccdc_plan_s &P, int k) { return P.node_nrounds[k] > 0; }
+bool is_local(const ccdc_plan_s &P, int k) { return k / (P.K / P.shard_world) == P.shard_rank; }
+bool has_part(const ccdc_plan_s &P, int k) { return P.nlocal[k] > 0 && is_local(P, k); }
+bool has_decoded(const ccdc_plan_s &P, int k) { return P.node_nrounds[k] > 0 && is_local(P, k); }
 
 int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *const *src, void *const *dst,
                   void *dst_single, const void *coded_in, int b, long long file_stride, cudaStream_t st) {
@@ -637,7 +644,7 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     if (plan->device != -1) return CCDC_ESTATE;
     struct Piece { const void *src; size_t bytes; const void **dst; };
     ccdc_gather_table *tabs[4] = {&plan->enc_fused, &plan->cmb, &plan->enc_pk, &plan->dec_pk};
-    Piece pieces[10];
+    Piece pieces[11];
     int np = 0;
     for (ccdc_gather_table *T : tabs) {
         pieces[np++] = {T->rows.data(), T->rows.size() * sizeof(ccdc_row), (const void **)&T->d_rows};
@@ -645,6 +652,7 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     }
     pieces[np++] = {plan->dec_terms.data(), plan->dec_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_dec_terms};
     pieces[np++] = {plan->red_terms.data(), plan->red_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_red_terms};
+    pieces[np++] = {plan->out_rows.data(), plan->out_rows.size() * sizeof(int), (const void **)&plan->d_out_rows};
     size_t total = 0;
     for (int i = 0; i < np; ++i) total += (pieces[i].bytes + 255) / 256 * 256;
     void *blob = nullptr;
@@ -666,6 +674,7 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
 }
 
 int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packets, void *stream) {
+    if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the stepwise API is single-GPU
     if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
@@ -677,6 +686,7 @@ int ccdc_combine(ccdc_plan_t *plan, const void *const *part, void *const *packet
 }
 
 int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void *stream) {
+    if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the stepwise API is single-GPU
     if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, packets, has_part);
@@ -688,6 +698,7 @@ int ccdc_encode(ccdc_plan_t *plan, const void *const *packets, void *coded, void
 
 int ccdc_decode(ccdc_plan_t *plan, const void *const *packets, const void *coded, void *const *decoded,
                 void *stream) {
+    if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the stepwise API is single-GPU
     if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !aligned16(coded)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, packets, has_part);
@@ -699,6 +710,7 @@ int ccdc_decode(ccdc_plan_t *plan, const void *const *packets, const void *coded
 }
 
 int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *decoded, void *out, void *stream) {
+    if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the stepwise API is single-GPU
     if (!plan || !out || !aligned16(out)) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
     if (rc == CCDC_OK) rc = check_ptr_array(*plan, decoded, has_decoded);
@@ -756,6 +768,8 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
     dp.ws = static_cast<uint32_t *>(workspace);
     dp.terms = P.d_dec_terms;
     dp.nout = P.J * P.K; dp.len = P.len; dp.s = P.s; dp.file_stride = P.row_elems;
+    dp.out_rows = P.shard_world > 1 ? P.d_out_rows : nullptr;
+    dp.nlist = P.shard_world > 1 ? (long long)P.out_rows.size() : dp.nout;
     dp.nterm = P.nterm; dp.terms_per_chunk = P.terms_per_chunk;
     dp.K = P.K; dp.r = P.r; dp.b = (int)P.b; dp.TS = P.term_stride; dp.nchunk = P.nchunk;
     const int stage_refs = 1024;                                    // 16 KiB of shared memory
@@ -765,7 +779,7 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         constexpr bool F32 = decltype(f32)::value;
         const long long tile = (long long)P.decode_threads * VEC * DUNROLL;
         dp.tiles_per_seg = (P.s + tile - 1) / tile;
-        const long long blocks = dp.nout * P.nchunk * P.r * dp.tiles_per_seg;
+        const long long blocks = dp.nlist * P.nchunk * P.r * dp.tiles_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
         // small r: the instantiation with r-1 as a compile-time constant
@@ -794,14 +808,16 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         }
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
-        const long long n = dp.nout * P.len;
-        k_sum_chunks<F32><<<(unsigned)((n + DTHREADS - 1) / DTHREADS), DTHREADS, 0, st>>>(dp.ws, dp.out, n, P.nchunk);
+        const long long n = dp.nout * P.len, todo = dp.nlist * P.len;
+        k_sum_chunks<F32><<<(unsigned)((todo + DTHREADS - 1) / DTHREADS), DTHREADS, 0, st>>>(
+            dp.ws, dp.out, dp.out_rows, dp.nlist, P.len, n, P.nchunk);
         return check_launch();
     });
 }
 
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out, void *workspace,
                  void *stream) {
+    if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the coded rows must be exchanged between the two launches
     if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
     if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
     int rc = ccdc_encode_fused(plan, part, coded, stream);

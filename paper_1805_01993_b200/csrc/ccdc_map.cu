@@ -598,7 +598,7 @@ encode_tiled_fn encode_tiled() {
 
 long long total_jobs(const ccdc_plan_s &P) {
     long long n = 0;
-    for (int k = 0; k < P.K; ++k) n += P.node_nfiles[k];
+    for (int k = 0; k < P.K; ++k) if (ccdc_plan_node_is_local(&P, k)) n += P.node_nfiles[k];
     return n;
 }
 
@@ -627,8 +627,9 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
     MapParams mp;
     std::memset(&mp, 0, sizeof(mp));
     for (int k = 0; k < P.K; ++k) {
-        mp.first_job[k + 1] = mp.first_job[k] + P.node_nfiles[k];
-        if (P.nlocal[k] == 0) continue;
+        const bool here = P.nlocal[k] > 0 && ccdc_plan_node_is_local(plan, k);
+        mp.first_job[k + 1] = mp.first_job[k] + (here ? P.node_nfiles[k] : 0);
+        if (!here) continue;
         if (!files_x[k] || !files_y[k] || !part[k]) return CCDC_EINVAL;
         if ((reinterpret_cast<uintptr_t>(files_x[k]) | reinterpret_cast<uintptr_t>(part[k])) & 15u) return CCDC_EINVAL;
         if (reinterpret_cast<uintptr_t>(files_y[k]) & 3u) return CCDC_EINVAL;

@@ -87,6 +87,67 @@ int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
     return CCDC_OK;
 }
 
+// split of the batch loop of the fused decode over `nout` output rows: enough
+// thread blocks to fill the GPU (148 SMs x 8 resident blocks) while a block
+// still walks a fair number of batches
+void choose_split(ccdc_plan_s &P, long long nout) {
+    // short segments: one large block per segment beats two smaller ones (measured on K=16, r=4)
+    P.decode_threads = CCDC_DECODE_THREADS;
+    if (P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
+        P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS)
+        P.decode_threads = CCDC_DECODE_THREADS_SHORT;
+    const long long tile = (long long)P.decode_threads * P.vec * CCDC_DECODE_VECTORS;
+    const long long tiles_per_seg = (P.s + tile - 1) / tile;
+    const long long base = std::max(1LL, nout * P.r * tiles_per_seg);
+    long long want = (148LL * 8 + base - 1) / base;
+    long long cap = std::max(1LL, P.nterm / 8);
+    long long nch = std::max(1LL, std::min(want, cap));
+    P.terms_per_chunk = (P.nterm + nch - 1) / nch;
+    P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
+}
+
+// Restrict a finished plan to the nodes of one rank out of `world` (node k lives
+// on rank k / (K/world)).  The rank encodes the coded rows its nodes send, into a
+// send buffer of its own; after an all-gather of the send buffers (rank-major)
+// coded row (round, a) sits at coded_row_pos; the rank decodes for its nodes.
+int apply_shard(ccdc_plan_s &P, int rank, int world) {
+    const int K = P.K, r = P.r;
+    if (world < 1 || rank < 0 || rank >= world || K % world != 0) return CCDC_EINVAL;
+    const int per = K / world;
+    const long long nrows = P.nround * (r + 1);
+    P.shard_rank = rank; P.shard_world = world;
+    P.coded_row_pos.assign(nrows, 0);
+    std::vector<long long> count(world, 0);
+    for (long long cr = 0; cr < nrows; ++cr) {
+        const int owner = P.round_group[cr] / per;          // round_group is [round][a] = sender of row cr
+        P.coded_row_pos[cr] = count[owner]++;
+    }
+    for (int w = 1; w < world; ++w) if (count[w] != count[0]) return CCDC_EINVAL;
+    P.send_rows = count[0];
+    for (long long cr = 0; cr < nrows; ++cr) P.coded_row_pos[cr] += (P.round_group[cr] / per) * P.send_rows;
+    // encode: only the rows this rank's nodes send, packed into its send buffer
+    ccdc_gather_table enc;
+    enc.na = P.enc_fused.na; enc.n_max = P.enc_fused.n_max;
+    for (long long cr = 0; cr < nrows; ++cr) {
+        if (P.round_group[cr] / per != rank) continue;
+        ccdc_row R = P.enc_fused.rows[cr];
+        R.dst_off = (P.coded_row_pos[cr] - rank * P.send_rows) * P.s_pad;
+        enc.rows.push_back(R);
+        for (int a = 0; a < enc.na; ++a) enc.refs.push_back(P.enc_fused.refs[(size_t)cr * enc.na + a]);
+    }
+    P.enc_fused = enc;
+    // decode: coded rows are found at their gathered positions
+    for (size_t x = 0; x < P.dec_terms.size(); x += P.term_stride) {
+        ccdc_ref &c = P.dec_terms[x];
+        if (c.off >= 0) c.off = P.coded_row_pos[c.off / P.s_pad] * P.s_pad;
+    }
+    P.out_rows.clear();
+    for (long long j = 0; j < P.J; ++j)
+        for (int k = rank * per; k < (rank + 1) * per; ++k) P.out_rows.push_back((int)(j * K + k));
+    choose_split(P, (long long)P.out_rows.size());
+    return CCDC_OK;
+}
+
 // everything that follows from batches + rounds
 int finish(ccdc_plan_s &P) {
     const int K = P.K, r = P.r;
@@ -234,23 +295,7 @@ int finish(ccdc_plan_s &P) {
             }
         }
 
-    // ---- split of the batch loop of the fused decode: enough thread blocks to
-    // fill the GPU (148 SMs x 8 resident blocks) while a block still walks a
-    // fair number of batches
-    {
-        // short segments: one large block per segment beats two smaller ones (measured on K=16, r=4)
-        if (P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
-            P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS)
-            P.decode_threads = CCDC_DECODE_THREADS_SHORT;
-        const long long tile = (long long)P.decode_threads * P.vec * CCDC_DECODE_VECTORS;
-        const long long tiles_per_seg = (P.s + tile - 1) / tile;
-        const long long base = nout * r * tiles_per_seg;
-        long long want = (148LL * 8 + base - 1) / base;
-        long long cap = std::max(1LL, P.nterm / 8);
-        long long nch = std::max(1LL, std::min(want, cap));
-        P.terms_per_chunk = (P.nterm + nch - 1) / nch;
-        P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
-    }
+    choose_split(P, nout);
 
     // ---- every offset must stay inside its buffer
     auto check_table = [&](const ccdc_gather_table &T, bool src_is_packets, bool dst_kind_coded,
@@ -446,6 +491,32 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
 }  // namespace
 
 extern "C" {
+
+int ccdc_plan_sharded(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, int jobs, int rank,
+                      int world, ccdc_plan_t **out) {
+    int rc = make_plan(K, r, N, Q, B, dtype, jobs != 0, out);
+    if (rc != CCDC_OK) return rc;
+    rc = apply_shard(**out, rank, world);
+    if (rc != CCDC_OK) { delete *out; *out = nullptr; }
+    return rc;
+}
+
+long long ccdc_plan_coded_row_position(const ccdc_plan_t *p, long long g, int a) {
+    if (!p || g < 0 || g >= p->nround || a < 0 || a > p->r) return -1;
+    const long long cr = g * (p->r + 1) + a;
+    return p->shard_world > 1 ? p->coded_row_pos[cr] : cr;
+}
+
+size_t ccdc_coded_send_bytes(const ccdc_plan_t *p) {
+    if (!p) return 0;
+    const long long rows = p->shard_world > 1 ? p->send_rows : p->nround * (p->r + 1);
+    return (size_t)(rows * p->s_pad) * 4;
+}
+
+int ccdc_plan_node_is_local(const ccdc_plan_t *p, int k) {
+    if (!p || k < 0 || k >= p->K) return 0;
+    return k / (p->K / p->shard_world) == p->shard_rank;
+}
 
 int ccdc_plan_compression(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
     return make_compression_plan(K, r, N, Q, B, dtype, out);

@@ -237,6 +237,49 @@ def test_compression_only_matches_oracle(ccdc, K, r, N, Q, B, dtype):
     assert e.value.status == ccdc.ESTATE
 
 
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B,world,jobs", [(4, 2, 12, 4, 300, 2, False), (6, 3, 40, 6, 2049, 3, False),
+                                                  (8, 3, 112, 8, 1024, 4, False), (10, 3, 480, 10, 512, 2, False),
+                                                  (4, 2, 6, 4, 100, 2, True), (6, 2, 9, 12, 64, 3, True)])
+def test_node_sharded_ranks_emulated_on_one_gpu(ccdc, K, r, N, Q, B, world, jobs, dtype):
+    """K/world logical nodes per GPU: every rank encodes the coded rows its nodes send,
+    the send buffers are gathered rank-major (here a concatenation stands in for the
+    all-gather; the ranks run one after the other, none waits for another), and every
+    rank decodes for its own nodes.  Coded rows and outputs against the oracle."""
+    full = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+    o = Oracle(K, r, N, Q, B, dtype, mode="paper" if jobs else "single")
+    v = values_numpy(full.J * N, Q, B, dtype, seed=K + world)
+    o.load_values(v)
+    o.shuffle()
+    vt = torch.from_numpy(v).cuda()
+    plans = [ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs, shard=(rk, world)) for rk in range(world)]
+    parts, sends = [], []
+    for pl in plans:
+        part = pl.alloc_partitions()
+        pl.fill_partitions(part, vt)
+        send_w, send = guarded(pl.coded_send_bytes // 4, pl.torch_dtype)
+        pl.encode_fused(part, send)
+        torch.cuda.synchronize()
+        assert canaries_intact(send_w, pl.coded_send_bytes // 4)
+        parts.append(part); sends.append(send)
+    coded = torch.cat(sends)                                  # the all-gather
+    assert coded.numel() * 4 == full.coded_bytes
+    s, sp = full.segment_elems, full.coded_row_elems
+    got = bits(coded).reshape(-1, sp)[:, :s]
+    ref = o.coded().reshape(-1, s)
+    order = [plans[0].coded_row_position(g, a) for g in range(full.num_groups) for a in range(r + 1)]
+    assert np.array_equal(got[order], ref)
+    out = torch.full((full.J * Q * B,), 7, dtype=full.torch_dtype, device="cuda")
+    for pl, part in zip(plans, parts):
+        ws = pl.alloc(pl.workspace_bytes)
+        pl.decode_reduce(part, coded, out, ws)
+    torch.cuda.synchronize()
+    assert_outputs(out, o, dtype)
+    with pytest.raises(ccdc.CcdcError) as e:
+        plans[0].shuffle(parts[0], coded, out, None)
+    assert e.value.status == ccdc.ESTATE
+
+
 def test_bad_arguments_are_refused(ccdc):
     plan = ccdc.Plan(4, 2, 12, 4, 64, "int32")
     part = plan.alloc_partitions()

@@ -142,3 +142,26 @@ def test_compression_plan(K, r, N):
     assert p.coded_bytes == 0 and p.workspace_bytes == 0
     with pytest.raises(ccdc.CcdcError):
         ccdc.Plan(5, 2, 11, 5, 8, "float32", compression=True)      # mu*N not an integer
+
+
+@pytest.mark.parametrize("K,r,N,world,jobs", [(4, 2, 12, 2, False), (6, 3, 40, 3, False), (8, 3, 112, 4, False),
+                                              (4, 2, 6, 2, True), (6, 2, 9, 3, True)])
+def test_node_sharded_plans_agree_on_the_gathered_layout(K, r, N, world, jobs):
+    """Every rank's plan places coded row (round, a) at the same position of the
+    gathered buffer; the rows a rank sends fill exactly its own slice, in order."""
+    Q, B = K, 8
+    plans = [ccdc.Plan(K, r, N, Q, B, "int32", jobs=jobs, shard=(rk, world)) for rk in range(world)]
+    full = ccdc.Plan(K, r, N, Q, B, "int32", jobs=jobs)
+    rows = full.num_groups * (r + 1)
+    pos = [[pl.coded_row_position(g, a) for g in range(full.num_groups) for a in range(r + 1)] for pl in plans]
+    assert all(p == pos[0] for p in pos) and sorted(pos[0]) == list(range(rows))
+    per = rows // world
+    for rk, pl in enumerate(plans):
+        assert pl.coded_send_bytes == per * pl.coded_row_elems * 4 and pl.coded_bytes == full.coded_bytes
+        mine = [pos[0][g * (r + 1) + a] for g in range(full.num_groups) for a, k in enumerate(full.group(g))
+                if k // (K // world) == rk]
+        assert mine == list(range(rk * per, (rk + 1) * per))
+        assert [pl.node_is_local(k) for k in range(K)] == [k // (K // world) == rk for k in range(K)]
+        assert pl.coded_bits == full.coded_bits        # what crosses between the GPUs is the multicast load
+    with pytest.raises(ccdc.CcdcError):
+        ccdc.Plan(6, 2, 15, 6, 8, "int32", shard=(0, 4))     # world must divide K

@@ -43,6 +43,43 @@ dist.destroy_process_group()
 """
 
 
+SHARD_WORKER = r"""
+import os, sys, json
+sys.path.insert(0, os.environ["CCDC_ROOT"])
+import numpy as np, torch, torch.distributed as dist
+from oracle.ccdc_oracle import Oracle
+from paper_1805_01993_b200 import build, ccdc
+from paper_1805_01993_b200.inputs import values_numpy
+
+dist.init_process_group("gloo")
+rank, world = dist.get_rank(), dist.get_world_size()
+build.build_library()
+K, r, N, Q, B = 6, 2, 15, 6, 20
+plan = ccdc.Plan(K, r, N, Q, B, "int32", shard=(rank, world))
+o = Oracle(K, r, N, Q, B, "int32")
+o.run(values_numpy(N, Q, B, "int32", seed=4))
+ref = o.coded()                                     # [round][sender rank][s]
+sp, s = plan.coded_row_elems, plan.segment_elems
+# what this rank's nodes send, in the order of the rank's send buffer (stand-in for the encode kernel)
+send = torch.zeros(plan.coded_send_bytes // 4, dtype=torch.int32).view(-1, sp)
+per = send.shape[0]
+for g in range(plan.num_groups):
+    for a, k in enumerate(plan.group(g)):
+        if plan.node_is_local(k):
+            send[plan.coded_row_position(g, a) - rank * per, :s] = torch.from_numpy(ref[g, a].view(np.int32))
+coded = torch.zeros(plan.coded_bytes // 4, dtype=torch.int32)
+dist.all_gather_into_tensor(coded, send.reshape(-1))        # the exchange between GPUs
+coded = coded.view(-1, sp)
+ok = all(np.array_equal(coded[plan.coded_row_position(g, a), :s].numpy().view(np.uint32), ref[g, a])
+         for g in range(plan.num_groups) for a in range(r + 1))
+flag = torch.tensor([1 if ok else 0])
+dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+if rank == 0:
+    print(json.dumps({"ok": int(flag.item()), "rows": int(coded.shape[0]), "send_rows": per}))
+dist.destroy_process_group()
+"""
+
+
 def run_two_ranks(script_args, env_extra=None):
     env = dict(os.environ, CCDC_ROOT=str(ROOT), MASTER_ADDR="127.0.0.1")
     env.update(env_extra or {})
@@ -62,6 +99,18 @@ def test_timing_protocol_and_independent_jobs(tmp_path):
     assert out["value"] == pytest.approx(2 * 1e9 / 5e-3 / 1e9)  # both ranks' bytes over the slowest time
     assert out["bits"][0] == out["bits"][1]                     # same scheme on every rank
     assert out["sums"][0] != out["sums"][1]                     # different synthetic inputs
+
+
+def test_node_sharded_exchange_over_a_real_all_gather(tmp_path):
+    """Two ranks, three logical nodes each: the rows each rank's nodes send (taken from
+    the oracle, standing in for the encode kernel) are all-gathered with gloo and
+    every coded row is found where the plan says the decode will look for it."""
+    script = tmp_path / "shard_worker.py"
+    script.write_text(SHARD_WORKER)
+    res = run_two_ranks([str(script)])
+    assert res.returncode == 0, res.stderr[-2000:]
+    out = json.loads([l for l in res.stdout.splitlines() if l.startswith("{")][-1])
+    assert out["ok"] == 1 and out["rows"] == 2 * out["send_rows"] == 20 * 3
 
 
 def test_reference_arm_runs_on_rank0_only():
