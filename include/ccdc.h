@@ -248,6 +248,18 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
 int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, void *stream);
 int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
                        void *workspace, void *stream);
+
+/* Encode fused with the exchange between GPUs (node-sharded plans only, else
+ * CCDC_ESTATE): the multicast of Section IV-B done by the producing kernel.
+ * peer_coded: HOST array of `world` device pointers, entry d = rank d's full
+ * coded buffer (ccdc_coded_bytes) as addressable from this GPU (its own buffer
+ * for d = this rank, peer mappings for the others).  Every coded row this rank's
+ * nodes send is stored straight into its gathered position in all `world`
+ * buffers, so no separate all-gather is needed; the ranks must still synchronise
+ * (on the host, or with stream events) before any of them launches
+ * ccdc_decode_reduce, because a kernel of one rank never waits for another
+ * rank.  Needs one file per batch or r <= 4 operands (CCDC_ESIZE otherwise). */
+int ccdc_encode_fused_peers(ccdc_plan_t *plan, const void *const *part, void *const *peer_coded, void *stream);
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out,
                  void *workspace, void *stream);
 

@@ -63,6 +63,7 @@ SIGNATURES = {
     "ccdc_reduce": (_I, [_P, _PP, _PP, _P, _P]),
     "ccdc_encode_fused": (_I, [_P, _PP, _P, _P]),
     "ccdc_decode_reduce": (_I, [_P, _PP, _P, _P, _P, _P]),
+    "ccdc_encode_fused_peers": (_I, [_P, _PP, _PP, _P]),
     "ccdc_shuffle": (_I, [_P, _PP, _P, _P, _P, _P]),
     "ccdc_static_scratch_bytes": (_SZ, []),
     "ccdc_decode_reduce_static": (_I, [_P, _PP, _P, _P, _P]),
@@ -308,6 +309,11 @@ class Plan:
     def encode_fused(self, part, coded, stream=None):
         _check(lib().ccdc_encode_fused(self._h, _ptr_array(part), coded.data_ptr(), _stream_handle(stream)),
                "ccdc_encode_fused")
+
+    def encode_fused_peers(self, part, peer_coded, stream=None):
+        """``peer_coded``: every rank's full coded buffer as addressable from this GPU."""
+        _check(lib().ccdc_encode_fused_peers(self._h, _ptr_array(part), _ptr_array(peer_coded),
+                                             _stream_handle(stream)), "ccdc_encode_fused_peers")
 
     def decode_reduce(self, part, coded, out, workspace=None, stream=None):
         ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None

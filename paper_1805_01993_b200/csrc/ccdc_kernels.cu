@@ -166,8 +166,10 @@ struct GatherParams {
     long long spans_per_row;
     long long span_elems;       // elements of a row one block covers (a multiple of the tile)
     long long file_stride;
+    long long dst_add;          // added to every row's destination offset
     int na;
     int b;
+    int replicas;               // > 0: every row is stored into dst[0..replicas-1] (peer buffers)
 };
 
 // position in a block's chunk sequence: for each tile of the span, the coded
@@ -286,7 +288,7 @@ k_gather_static(const __grid_constant__ GatherParams p) {
 #pragma unroll
     for (int a = 0; a < RS; ++a) E[a] = p.refs[row * RS + a];
     const uint32_t *src = p.src[R.src_node];
-    uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
+    uint32_t *dst = p.dst[p.replicas > 0 ? 0 : R.dst_node] + R.dst_off + p.dst_add;
     for (long long base = begin; base < end; base += TILE) {
         Words<VEC> v[RS][SUNROLL];
 #pragma unroll
@@ -316,7 +318,13 @@ k_gather_static(const __grid_constant__ GatherParams p) {
             const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
 #pragma unroll
             for (int a = 1; a < RS; ++a) xor_into<VEC>(v[0][u], v[a][u]);
-            if (j < end) store_words<VEC>(dst + j, v[0][u]);
+            if (j < end) {
+                store_words<VEC>(dst + j, v[0][u]);
+                // the same row into every other peer's buffer (plain stores over NVLink when the
+                // pointers are peer mappings): the all-gather happens as the rows are produced
+                for (int d = 1; d < p.replicas; ++d)
+                    store_words<VEC>(p.dst[d] + R.dst_off + p.dst_add + j, v[0][u]);
+            }
         }
     }
 }
@@ -557,13 +565,19 @@ bool has_part(const ccdc_plan_s &P, int k) { return P.nlocal[k] > 0 && is_local(
 bool has_decoded(const ccdc_plan_s &P, int k) { return P.node_nrounds[k] > 0 && is_local(P, k); }
 
 int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *const *src, void *const *dst,
-                  void *dst_single, const void *coded_in, int b, long long file_stride, cudaStream_t st) {
+                  void *dst_single, const void *coded_in, int b, long long file_stride, cudaStream_t st,
+                  void *const *peers = nullptr, int npeers = 0, long long dst_add = 0) {
     if (T.rows.empty() || T.n_max == 0) return CCDC_OK;
     GatherParams gp;
     std::memset(&gp, 0, sizeof(gp));
     for (int k = 0; k < P.K; ++k) {
         gp.src[k] = static_cast<const uint32_t *>(src[k]);
         gp.dst[k] = static_cast<uint32_t *>(dst_single ? dst_single : dst[k]);
+    }
+    if (npeers > 0) {
+        for (int d = 0; d < npeers; ++d) gp.dst[d] = static_cast<uint32_t *>(peers[d]);
+        gp.replicas = npeers;
+        gp.dst_add = dst_add;
     }
     gp.coded_in = static_cast<const uint32_t *>(coded_in);
     gp.rows = T.d_rows; gp.refs = T.d_refs;
@@ -573,6 +587,7 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
         const bool lean = !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
+        if (npeers > 0 && !lean) return CCDC_ESIZE;         // peer stores exist in the lean kernel only
         const long long tile = lean ? (long long)STHREADS * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 148 SMs x 16 blocks
@@ -748,6 +763,21 @@ int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, v
     if (rc != CCDC_OK) return rc;
     return launch_gather(*plan, plan->enc_fused, part, nullptr, coded, nullptr, (int)plan->b, plan->row_elems,
                          static_cast<cudaStream_t>(stream));
+}
+
+int ccdc_encode_fused_peers(ccdc_plan_t *plan, const void *const *part, void *const *peer_coded, void *stream) {
+    if (!plan || !peer_coded) return CCDC_EINVAL;
+    if (plan->compression_mode || plan->shard_world < 2) return CCDC_ESTATE;
+    if (plan->shard_world > CCDC_MAX_K) return CCDC_ESIZE;
+    for (int d = 0; d < plan->shard_world; ++d)
+        if (!peer_coded[d] || !aligned16(peer_coded[d])) return CCDC_EINVAL;
+    int rc = check_ptr_array(*plan, part, has_part);
+    if (rc == CCDC_OK) rc = ensure_device(plan);
+    if (rc != CCDC_OK) return rc;
+    // this rank's rows go to their gathered position in every rank's buffer
+    return launch_gather(*plan, plan->enc_fused, part, nullptr, peer_coded[0], nullptr, (int)plan->b, plan->row_elems,
+                         static_cast<cudaStream_t>(stream), peer_coded, plan->shard_world,
+                         (long long)plan->shard_rank * plan->send_rows * plan->s_pad);
 }
 
 int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,

@@ -278,6 +278,21 @@ def test_node_sharded_ranks_emulated_on_one_gpu(ccdc, K, r, N, Q, B, world, jobs
     with pytest.raises(ccdc.CcdcError) as e:
         plans[0].shuffle(parts[0], coded, out, None)
     assert e.value.status == ccdc.ESTATE
+    # the encode that stores straight into every rank's buffer (here: `world` buffers on one GPU)
+    if r <= 4:
+        guards = [guarded(full.coded_bytes // 4, full.torch_dtype) for _ in range(world)]
+        peers = [gview for _, gview in guards]
+        for pl, part in zip(plans, parts):
+            pl.encode_fused_peers(part, peers)
+        torch.cuda.synchronize()                              # stands in for the ranks' synchronisation
+        for whole, gview in guards:
+            assert canaries_intact(whole, full.coded_bytes // 4)
+            assert np.array_equal(bits(gview).reshape(-1, sp)[:, :s], got)
+        out2 = torch.full_like(out, 7)
+        for rk, (pl, part) in enumerate(zip(plans, parts)):
+            pl.decode_reduce(part, peers[rk], out2, pl.alloc(pl.workspace_bytes))
+        torch.cuda.synchronize()
+        assert torch.equal(out2, out)
 
 
 def test_bad_arguments_are_refused(ccdc):
