@@ -275,7 +275,7 @@ def run_ours(args, w):
         wvec = torch.randn(d, generator=gen, device=dev).to(torch.bfloat16)
         map_ws = torch.empty(plan.map_workspace_bytes(w.map_rows) // 4, dtype=torch.float32, device=dev)
         map_bytes = sum(t.numel() * 2 for t in files_x) + sum(plan.partition_bytes(k) for k in range(w.K))
-        stages.append(("k_map_residual+k_map_gradient",
+        stages.append(("k_map",
                        lambda: plan.map(files_x, files_y, wvec, w.map_rows, part, map_ws)))
     else:
         # every rank is an independent job of the same shape: its own seed
@@ -289,7 +289,7 @@ def run_ours(args, w):
         stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, coded)))
     stages.append(("k_decode_reduce", lambda: plan.decode_reduce(part, coded, out, ws)))
     share = world if sharded else 1                      # a rank's part of the job
-    stage_bytes = {"k_map_residual+k_map_gradient": map_bytes, "k_gather(encode)": by["encode_kernel"] // share,
+    stage_bytes = {"k_map": map_bytes, "k_gather(encode)": by["encode_kernel"] // share,
                    "k_decode_reduce": by["decode_kernel"] // share,
                    "all_gather(coded rows)": by["coded_write"] * (world - 1) // max(world, 1)}
     input_bytes = sum(plan.partition_bytes(k) for k in range(w.K)) + map_bytes
@@ -405,6 +405,7 @@ def run_ours(args, w):
                    "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
                           f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written between steps, steps timed one by one"),
                    "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": plan.J,
+                   **({"map_kernel": ccdc.map_last_kernel()} if w.map_rows else {}),
                    "load_per_JQT": plan.coded_bits / (plan.J * w.Q * 32 * w.B),
                    "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
                    "algorithmic_bytes_per_step": by["total"] + map_bytes,

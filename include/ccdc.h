@@ -189,13 +189,29 @@ size_t ccdc_workspace_bytes(const ccdc_plan_t *plan);         /* ccdc_shuffle sc
  *   (residuals plus a few control words; the call resets what it needs).
  * F32 plans only (CCDC_ESTATE otherwise).  CCDC_ESIZE unless rows is a multiple
  * of 16 in 16..4096 and d a multiple of 512 up to 65536.  Asynchronous on
- * `stream`: one memset and ONE kernel launch.  Inside it, work items are handed
- * out in order by an atomic ticket (per file its first-product blocks, then the
- * second-product blocks of the previous file) so that the second product finds
- * the file in L2; a second-product block polls a per-file counter until the
- * file's residuals are complete.  The blocks it waits for hold smaller tickets,
- * are therefore already running and wait on nothing, so the poll always ends;
- * it is bounded anyway, and ccdc_map_status reports if a bound was ever hit.
+ * `stream`: one memset and one or two kernel launches.
+ *
+ * Which kernel runs (ccdc_map_last_kernel tells):
+ *  - d = 2048, 4096, 8192 or 16384: a thread-block cluster of d/2048 blocks owns a
+ *    file, each block 2048 columns.  X is staged by TMA into a ring of
+ *    shared-memory stages (8 rows x 2048 columns each) and read from HBM exactly
+ *    once: both products of a row block run from the same stage, the blocks of a
+ *    cluster exchanging their partial dot products through distributed shared
+ *    memory.  Files are cut into units of rows/4 rows (when rows is a multiple of
+ *    32) that are shared out evenly over the clusters; a file's gradient is always
+ *    ((unit0 + unit1) + unit2) + unit3, whichever clusters computed the units, so
+ *    replicas stay bit-identical; files cut between two clusters are summed by a
+ *    small second launch from the workspace.  All waits (mbarrier polls) are
+ *    bounded.
+ *  - other shapes, or a device or driver without tensor maps or room for the
+ *    cluster: loads through registers; work items are handed out in order by an
+ *    atomic ticket (per file its first-product blocks, then the second-product
+ *    blocks of an earlier file) so that the second product finds the file in L2;
+ *    a second-product block polls a per-file counter until the file's residuals
+ *    are complete.  The blocks it waits for hold smaller tickets, are therefore
+ *    already running and wait on nothing, so the poll always ends; it is bounded
+ *    anyway.
+ * ccdc_map_status reports if a bound was ever hit in either kernel.
  *
  * ccdc_map_status: call after the stream has been synchronised; copies one word
  * back (synchronous) and returns CCDC_OK, or CCDC_ESTATE if a wait ran out (the
@@ -204,6 +220,10 @@ size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows);
 int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
              long long rows, void *const *part, void *workspace, void *stream);
 int ccdc_map_status(const ccdc_plan_t *plan, long long rows, const void *workspace);
+/* Name of the kernel the most recent ccdc_map of this process launched ("k_map_cluster": X staged by
+ * TMA through a thread-block cluster, read once; "k_map": loads through registers, for shapes or
+ * devices the first cannot serve; "" before the first call).  Static string, not thread safe. */
+const char *ccdc_map_last_kernel(void);
 
 /* Pre-combining (Section IV-B): packets[k][local batch][t] = concatenation over
  * q in S_t of  sum_{n in batch} v_{q,n}, files added in ascending order

@@ -57,6 +57,7 @@ SIGNATURES = {
     "ccdc_map_workspace_bytes": (_SZ, [_P, _LL]),
     "ccdc_map": (_I, [_P, _PP, _PP, _P, _LL, _PP, _P, _P]),
     "ccdc_map_status": (_I, [_P, _LL, _P]),
+    "ccdc_map_last_kernel": (ctypes.c_char_p, []),
     "ccdc_combine": (_I, [_P, _PP, _PP, _P]),
     "ccdc_encode": (_I, [_P, _PP, _P, _P]),
     "ccdc_decode": (_I, [_P, _PP, _P, _PP, _P]),
@@ -344,3 +345,8 @@ class Plan:
 
 def num_kernel_launches() -> int:
     return lib().ccdc_num_kernel_launches()
+
+
+def map_last_kernel() -> str:
+    """Name of the kernel the most recent ``Plan.map`` launched."""
+    return lib().ccdc_map_last_kernel().decode()

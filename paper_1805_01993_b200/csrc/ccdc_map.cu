@@ -21,6 +21,7 @@
 #include <cstring>
 
 #include "ccdc_internal.h"
+#include "ccdc_map_cluster.h"
 
 namespace {
 
@@ -596,6 +597,8 @@ encode_tiled_fn encode_tiled() {
     return fn;
 }
 
+const char *last_kernel = "";       // which kernel the last ccdc_map launched (reported, not synchronised)
+
 long long total_jobs(const ccdc_plan_s &P) {
     long long n = 0;
     for (int k = 0; k < P.K; ++k) if (ccdc_plan_node_is_local(&P, k)) n += P.node_nfiles[k];
@@ -607,6 +610,15 @@ long long total_jobs(const ccdc_plan_s &P) {
 size_t residual_bytes(long long jobs, long long rows) { return ((size_t)(jobs * rows) * 4 + 255) / 256 * 256; }
 size_t control_bytes(long long jobs) { return ((size_t)(jobs + 2) * 4 + 255) / 256 * 256; }
 
+// Which kernel maps a shape: the cluster kernel (X read once, staged by TMA) where it fits, unless
+// the library was built with -DCCDC_MAP_USE_CLUSTER=0 or with the per-warp TMA variant.
+#ifndef CCDC_MAP_USE_CLUSTER
+#define CCDC_MAP_USE_CLUSTER (!CCDC_MAP_USE_TMA)
+#endif
+size_t pieces_bytes(long long jobs, long long rows, long long d) {
+    return CCDC_MAP_USE_CLUSTER ? ccdc_map_cluster_pieces_bytes(jobs, rows, d) : 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -614,7 +626,7 @@ extern "C" {
 size_t ccdc_map_workspace_bytes(const ccdc_plan_t *plan, long long rows) {
     if (!plan || rows <= 0) return 0;
     const long long jobs = total_jobs(*plan);
-    return residual_bytes(jobs, rows) + control_bytes(jobs);
+    return residual_bytes(jobs, rows) + control_bytes(jobs) + pieces_bytes(jobs, rows, plan->row_elems);
 }
 
 int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *files_y, const void *w,
@@ -650,6 +662,13 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     cudaError_t e = cudaMemsetAsync(control, 0, control_bytes(njobs), st);
     if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+#if CCDC_MAP_USE_CLUSTER
+    if (ccdc_map_cluster_fits(rows, d)) {
+        void *pieces = static_cast<char *>(workspace) + residual_bytes(njobs, rows) + control_bytes(njobs);
+        const int rc = ccdc_map_cluster_launch(P, files_x, files_y, w, rows, part, mp.first_job, pieces, mp.status, stream);
+        if (rc != 1) { last_kernel = "k_map_cluster"; return rc; }
+    }
+#endif
     int dev = 0, sms = 0, per_sm = 0;
     e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -679,6 +698,7 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
             if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
             if (per_sm >= 1) {
                 per_sm = std::min(per_sm, CCDC_MAP_BLOCKS_PER_SM);
+                last_kernel = "k_map_tma";
                 k_map_tma<<<(unsigned)(sms * per_sm), MAP_THREADS, smem, st>>>(tp);
                 ccdc_internal_count_launch();
                 e = cudaGetLastError();
@@ -696,11 +716,14 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_map, MAP_THREADS, smem);
     if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
     per_sm = std::max(1, std::min(per_sm, CCDC_MAP_BLOCKS_PER_SM));
+    last_kernel = "k_map";
     k_map<<<(unsigned)(sms * per_sm), MAP_THREADS, smem, st>>>(mp);
     ccdc_internal_count_launch();
     e = cudaGetLastError();
     return e == cudaSuccess ? CCDC_OK : ccdc_internal_cuda_fail((int)e);
 }
+
+const char *ccdc_map_last_kernel(void) { return last_kernel; }
 
 int ccdc_map_status(const ccdc_plan_t *plan, long long rows, const void *workspace) {
     if (!plan || !workspace || rows <= 0) return CCDC_EINVAL;

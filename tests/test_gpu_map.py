@@ -105,17 +105,27 @@ def run_job(ccdc, K, r, N, Q, B, rows, seed):
 def test_map_small(ccdc):
     worst = run_job(ccdc, 4, 2, 12, 4, 128, rows=32, seed=7)
     assert worst < 1e-5
+    assert ccdc.map_last_kernel() == "k_map"        # d = 512: served by the register kernel
 
 
 def test_map_wide_files(ccdc):
-    # d = 2048 columns, 48 rows, r = K-1
+    # d = 2048 columns, 48 rows, r = K-1: the smallest shape of the cluster kernel (one block per cluster)
     run_job(ccdc, 4, 3, 8, 4, 512, rows=48, seed=8)
+    assert ccdc.map_last_kernel() == "k_map_cluster"
+
+
+def test_map_cluster_of_two_with_split_files(ccdc):
+    # d = 4096 (clusters of two blocks), 128 rows = 4 units per file, 24 Map executions: with more
+    # clusters than files every file is cut over several clusters and summed by the combine pass
+    run_job(ccdc, 4, 2, 12, 4, 1024, rows=128, seed=10)
+    assert ccdc.map_last_kernel() == "k_map_cluster"
 
 
 def test_cfg5_full_job(ccdc):
     w = CONFIGS["cfg5"]
     worst = run_job(ccdc, w.K, w.r, w.N, w.Q, w.B, rows=w.map_rows, seed=9)
     assert worst < 1e-5
+    assert ccdc.map_last_kernel() == "k_map_cluster"
 
 
 TMA_VARIANT = r"""
@@ -131,6 +141,28 @@ t.run_job(ccdc, 4, 3, 8, 4, 512, rows=48, seed=8)
 t.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)
 print("tma variant ok")
 """
+
+
+REGISTER_VARIANT = TMA_VARIANT.replace('"libccdc_tma.so", ("CCDC_MAP_USE_TMA=1",)', '"libccdc_reg.so", ("CCDC_MAP_USE_CLUSTER=0",)') \
+    .replace("t.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)",
+             't.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)\nassert ccdc.map_last_kernel() == "k_map"') \
+    .replace("tma variant ok", "register variant ok")
+
+
+def test_register_kernel_on_cluster_shapes(ccdc, tmp_path):
+    """The register kernel is the fallback for devices that cannot run the cluster kernel: built
+    with the cluster kernel switched off, it is held to the same parity on the shapes the cluster
+    kernel normally takes."""
+    import subprocess
+    import sys
+    from pathlib import Path
+
+    root = Path(__file__).resolve().parent.parent
+    script = tmp_path / "register_variant.py"
+    script.write_text(REGISTER_VARIANT)
+    res = subprocess.run([sys.executable, str(script), str(root), str(tmp_path)], capture_output=True, text=True,
+                         timeout=900)
+    assert res.returncode == 0 and "register variant ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
 
 
 def test_tma_variant_of_the_map(ccdc, tmp_path):
