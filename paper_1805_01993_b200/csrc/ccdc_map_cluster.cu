@@ -59,6 +59,7 @@ constexpr int STAGE_BYTES = CHUNKS_CTA * RB * 128;  // 32 KiB
 constexpr int STAGES = 6;
 constexpr int XBUF = 4;                             // exchange buffers: a peer may run up to 3 row blocks ahead
 constexpr int MAX_CLUSTER = 8;
+constexpr int MAX_SPLIT = 160;                      // listed files cut between two shares (at most one per share)
 constexpr int WAIT_LIMIT = 1 << 20;
 
 struct ClusterParams {
@@ -71,6 +72,8 @@ struct ClusterParams {
     int *status;
     long long njobs, rows, d;
     int K, UF, nclusters;
+    int nsplit;                         // files cut between shares, listed below; -1: not listed, look at every file
+    int split_jobs[MAX_SPLIT];
 };
 
 __device__ __forceinline__ unsigned smem_u32(const void *ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
@@ -437,7 +440,7 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
 // Files whose units fell into two or more shares: out = ((piece 0 + unit b0) + unit b0+1) + ..., where
 // piece 0 is the sum of units 0 .. b0-1 left by the share that held the file's first unit.
 __global__ void k_map_combine(const __grid_constant__ ClusterParams p) {
-    const long long job = blockIdx.x;
+    const long long job = p.nsplit >= 0 ? p.split_jobs[blockIdx.x] : blockIdx.x;
     const long long units = p.njobs * p.UF, first = job * p.UF;
     const int c0 = share_of_unit(units, p.nclusters, first);
     if (c0 == share_of_unit(units, p.nclusters, first + p.UF - 1)) return;     // mapped whole by one share
@@ -545,12 +548,23 @@ int ccdc_map_cluster_launch(const ccdc_plan_s &P, const void *const *files_x, co
     if (resident < 1) return 1;
     const long long units = cp.njobs * cp.UF;
     cp.nclusters = (int)std::min<long long>(resident, units);
+    // the files whose units fall into two or more shares (a share boundary inside the file)
+    cp.nsplit = 0;
+    for (int c = 1; c < cp.nclusters && cp.nsplit >= 0; ++c) {
+        const long long ub = share_start(units, cp.nclusters, c);
+        if (ub % cp.UF == 0) continue;
+        const int job = (int)(ub / cp.UF);
+        if (cp.nsplit > 0 && cp.split_jobs[cp.nsplit - 1] == job) continue;
+        if (cp.nsplit == MAX_SPLIT) cp.nsplit = -1;
+        else cp.split_jobs[cp.nsplit++] = job;
+    }
     cfg.gridDim = dim3((unsigned)(cp.nclusters * C), 1, 1);
     e = cudaLaunchKernelEx(&cfg, k_map_cluster, cp);
     if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
     ccdc_internal_count_launch();
-    if (cp.nclusters > 1 && cp.UF > 1) {
-        k_map_combine<<<dim3((unsigned)cp.njobs, 8), 256, 0, cfg.stream>>>(cp);
+    if (cp.nsplit != 0) {
+        const unsigned nblocks = cp.nsplit > 0 ? (unsigned)cp.nsplit : (unsigned)cp.njobs;
+        k_map_combine<<<dim3(nblocks, 8), 256, 0, cfg.stream>>>(cp);
         ccdc_internal_count_launch();
         e = cudaGetLastError();
         if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
