@@ -156,12 +156,18 @@ def oracle_sample_shape(w, target_seconds):
     ``target_seconds`` on one core; calibrated on a very short value first."""
     from oracle.ccdc_oracle import Oracle
 
+    per_elem = None
     probe_B = w.r * 64
-    o = Oracle(w.K, w.r, w.N, w.Q, probe_B, w.dtype, mode="paper" if w.jobs else "single")
-    o.load_values(values_numpy(o.J * w.N, w.Q, probe_B, w.dtype, std=w.std))
-    t0 = time.perf_counter()
-    o.shuffle(); o.reduce()
-    per_elem = (time.perf_counter() - t0) / probe_B
+    for _ in range(2):      # second pass: a value long enough to leave the caches, about a second of work
+        o = Oracle(w.K, w.r, w.N, w.Q, probe_B, w.dtype, mode="paper" if w.jobs else "single")
+        o.load_values(values_numpy(o.J * w.N, w.Q, probe_B, w.dtype, std=w.std))
+        t0 = time.perf_counter()
+        o.shuffle(); o.reduce()
+        per_elem = (time.perf_counter() - t0) / probe_B
+        nxt = int(min(1.0, target_seconds) / per_elem) // (4 * w.r) * (4 * w.r)
+        if nxt <= probe_B or nxt >= w.B:
+            break
+        probe_B = nxt
     B = int(target_seconds / per_elem) // (4 * w.r) * (4 * w.r)
     return max(4 * w.r, min(B, w.B))
 
