@@ -105,9 +105,14 @@ __device__ __forceinline__ Words<VEC> batch_sum(const uint32_t *src, long long o
     if (j >= vl) return zero_words<VEC>();
     const uint32_t *p = src + off + j;
     Words<VEC> acc = load_words<VEC>(p);
-    for (int f = 1; f < b; ++f) {
-        p += file_stride;
-        add_into<VEC, F32>(acc, load_words<VEC>(p));
+    for (int f = 1; f < b; f += 4) {        // up to four files' loads in flight, added in file order
+        Words<VEC> w[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+            if (f + x < b) w[x] = load_words<VEC>(p + (long long)(f + x) * file_stride);
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+            if (f + x < b) add_into<VEC, F32>(acc, w[x]);
     }
     return acc;
 }
@@ -298,20 +303,29 @@ k_gather_static(const __grid_constant__ GatherParams p) {
                 const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
                 v[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + j) : zero_words<VEC>();
             }
-        for (int f = 1; !B1 && f < p.b; ++f) {      // the other files of each batch, ascending
-            Words<VEC> w[RS][SUNROLL];
+        // the other files of each batch, ascending; the loads of FU files are issued together
+        constexpr int FU = RS * SUNROLL >= 6 ? 2 : (RS * SUNROLL >= 3 ? 4 : 8);
+        for (int f = 1; !B1 && f < p.b; f += FU) {
+            Words<VEC> w[FU][RS][SUNROLL];
 #pragma unroll
-            for (int a = 0; a < RS; ++a)
+            for (int x = 0; x < FU; ++x)
 #pragma unroll
-                for (int u = 0; u < SUNROLL; ++u) {
-                    const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
-                    w[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + f * p.file_stride + j)
-                                                       : zero_words<VEC>();
+                for (int a = 0; a < RS; ++a)
+#pragma unroll
+                    for (int u = 0; u < SUNROLL; ++u) {
+                        const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+                        w[x][a][u] = (f + x < p.b && j < end && j < E[a].vl)
+                                         ? load_words<VEC>(src + E[a].off + (f + x) * p.file_stride + j)
+                                         : zero_words<VEC>();
+                    }
+#pragma unroll
+            for (int x = 0; x < FU; ++x)
+                if (f + x < p.b) {
+#pragma unroll
+                    for (int a = 0; a < RS; ++a)
+#pragma unroll
+                        for (int u = 0; u < SUNROLL; ++u) add_into<VEC, F32>(v[a][u], w[x][a][u]);
                 }
-#pragma unroll
-            for (int a = 0; a < RS; ++a)
-#pragma unroll
-                for (int u = 0; u < SUNROLL; ++u) add_into<VEC, F32>(v[a][u], w[a][u]);
         }
 #pragma unroll
         for (int u = 0; u < SUNROLL; ++u) {
