@@ -128,6 +128,21 @@ def test_cfg5_full_job(ccdc):
     assert ccdc.map_last_kernel() == "k_map_cluster"
 
 
+@pytest.mark.parametrize("K,r,N,Q,B,rows", [
+    (4, 2, 12, 4, 512, 32),      # d = 2048, one block per cluster, one row block per cluster (shortest pipeline)
+    (4, 2, 12, 4, 512, 64),      # d = 2048, two row blocks per unit, every file cut over four clusters
+    (4, 2, 12, 4, 2048, 48),     # d = 8192, clusters of four, rows not a multiple of 32: one unit per file
+    (4, 2, 12, 4, 4096, 32),     # d = 16384, clusters of eight
+    (4, 3, 4, 4, 512, 4096),     # the longest files the call accepts
+    (6, 2, 15, 6, 1024, 160),    # d = 6144 is not a cluster shape: register kernel
+])
+def test_map_cluster_shapes(ccdc, K, r, N, Q, B, rows):
+    worst = run_job(ccdc, K, r, N, Q, B, rows=rows, seed=11 + rows)
+    assert worst < 1e-5
+    d = Q * B
+    assert ccdc.map_last_kernel() == ("k_map_cluster" if d in (2048, 4096, 8192, 16384) else "k_map")
+
+
 TMA_VARIANT = r"""
 import sys
 sys.path.insert(0, sys.argv[1])
