@@ -91,19 +91,32 @@ int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
 // thread blocks to fill the GPU (148 SMs x 8 resident blocks) while a block
 // still walks a fair number of batches
 void choose_split(ccdc_plan_s &P, long long nout) {
-    // short segments: one large block per segment beats two smaller ones (measured on K=16, r=4)
+    auto split_for = [&](int threads, long long &per_chunk, int &nchunk) {
+        const long long tile = (long long)threads * P.vec * CCDC_DECODE_VECTORS;
+        const long long tiles_per_seg = (P.s + tile - 1) / tile;
+        const long long base = std::max(1LL, nout * P.r * tiles_per_seg);
+        const long long want = (148LL * 8 + base - 1) / base;
+        const long long cap = std::max(1LL, P.nterm / 8);
+        const long long nch = std::max(1LL, std::min(want, cap));
+        per_chunk = (P.nterm + nch - 1) / nch;
+        nchunk = (int)((P.nterm + per_chunk - 1) / per_chunk);
+        return base * nchunk;                       // thread blocks of the launch
+    };
     P.decode_threads = CCDC_DECODE_THREADS;
+    split_for(P.decode_threads, P.terms_per_chunk, P.nchunk);
+    // short segments: one large block per segment instead of two smaller ones, but only when the launch
+    // still has many waves of them (one such block is resident per SM); measured: K=16, r=4 gains 0.6 %,
+    // K=10, r=3 with 450 blocks would lose 17 %
     if (P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
-        P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS)
-        P.decode_threads = CCDC_DECODE_THREADS_SHORT;
-    const long long tile = (long long)P.decode_threads * P.vec * CCDC_DECODE_VECTORS;
-    const long long tiles_per_seg = (P.s + tile - 1) / tile;
-    const long long base = std::max(1LL, nout * P.r * tiles_per_seg);
-    long long want = (148LL * 8 + base - 1) / base;
-    long long cap = std::max(1LL, P.nterm / 8);
-    long long nch = std::max(1LL, std::min(want, cap));
-    P.terms_per_chunk = (P.nterm + nch - 1) / nch;
-    P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
+        P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS) {
+        long long per_chunk = 0;
+        int nchunk = 0;
+        if (split_for(CCDC_DECODE_THREADS_SHORT, per_chunk, nchunk) >= 148LL * 6) {
+            P.decode_threads = CCDC_DECODE_THREADS_SHORT;
+            P.terms_per_chunk = per_chunk;
+            P.nchunk = nchunk;
+        }
+    }
 }
 
 // Restrict a finished plan to the nodes of one rank out of `world` (node k lives
