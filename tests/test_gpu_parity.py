@@ -133,6 +133,10 @@ SHAPES = [
     (12, 6, 924, 12, 8),                    # 924 batches, 792 rounds of 7
     (9, 5, 252, 9, 1030),                   # r = 5: general (run-time r) decode path, b = 2
     (6, 2, 15, 6, 40000),                   # b = 1, long values: lean gather + deep-load decode
+    (4, 2, 54, 4, 1100),                    # b = 9: batch sums in groups of four files plus a remainder
+    (3, 1, 30, 3, 2100),                    # b = 10, r = 1: one operand, eight files' loads in flight
+    (5, 3, 50, 5, 777),                     # b = 5, three operands
+    (5, 4, 15, 5, 1300),                    # b = 3, four operands
 ]
 
 
@@ -144,7 +148,7 @@ def test_single_job_matches_oracle(ccdc, K, r, N, Q, B, dtype):
 
 @pytest.mark.parametrize("dtype", ["int32", "float32"])
 @pytest.mark.parametrize("K,r,N,Q,B", [(4, 2, 6, 4, 8), (5, 2, 9, 5, 37), (5, 3, 8, 10, 6), (6, 1, 6, 6, 5),
-                                       (6, 4, 10, 6, 4100)])
+                                       (6, 4, 10, 6, 4100), (5, 2, 21, 5, 2060)])     # the last: 7 files per batch
 def test_jobs_plan_matches_oracle(ccdc, K, r, N, Q, B, dtype):
     """The scheme as stated for J = C(K, r+1) jobs (stages 1 and 2)."""
     run_case(ccdc, K, r, N, Q, B, dtype, jobs=True, seed=3)
