@@ -18,8 +18,9 @@
 //   3. second product: each warp multiplies the three terms (A rows 0..2) by the
 //      transposed slab (ldmatrix.trans, mma.sync m16n8k8) and accumulates its
 //      256 gradient columns in registers.
-// The loop is software pipelined: the first product runs two row blocks ahead of
-// the second, so the exchange of a row block has a whole iteration to land.
+// The loop is software pipelined behind one block barrier per row block: the
+// first product runs two row blocks ahead of the second, a row block's partial
+// dots are sent in the iteration that computes them and received in the next.
 // The slab is read from shared memory twice and from HBM once.
 //
 // Summation order.  A file is cut into UF units of rows/UF rows (UF = 4 when
@@ -121,6 +122,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity, int li
     }
     return false;
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ unsigned peer_addr(unsigned local, unsigned rank) {
     unsigned remote;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(rank));
@@ -130,6 +134,10 @@ __device__ __forceinline__ unsigned peer_addr(unsigned local, unsigned rank) {
 __device__ __forceinline__ void peer_store(unsigned remote, float v, unsigned remote_bar) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
                  ::"r"(remote), "r"(__float_as_uint(v)), "r"(remote_bar) : "memory");
+}
+// block barrier of the compute, receive and fetch warps (the send warp does not take part)
+__device__ __forceinline__ void block_sync() {
+    asm volatile("bar.sync 1, %0;" ::"n"(THREADS - 32) : "memory");
 }
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -196,6 +204,7 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
     extern __shared__ unsigned char sh_raw[];
     __shared__ __align__(8) uint64_t full[STAGES];      // the stage's slab has landed
     __shared__ __align__(8) uint64_t xbar[XBUF];        // all blocks' partial dots of a row block have landed
+    __shared__ __align__(8) uint64_t pbar[4];           // the 8 warps' partial dots of a row block are in sh_part
     __shared__ float sh_part[4][WARPS][RB];
     __shared__ float xch[XBUF][MAX_CLUSTER][RB];
     __shared__ uint32_t sh_u[2][3][RB / 2];             // hi / mid / lo terms of u as bf16 pairs, two row blocks
@@ -210,6 +219,7 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
         for (int s = 0; s < XBUF; ++s) mbar_init(&xbar[s], 1);
+        for (int s = 0; s < 4; ++s) mbar_init(&pbar[s], WARPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -239,9 +249,9 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
         };
         if (lane == 0)
             while (nload < STAGES && nload < nrb) fetch();
-        __syncthreads();
+        block_sync();
         for (long long i = 0; i < nrb; ++i) {
-            __syncthreads();    // the second product of row block i-1 is over: its stage can be refilled
+            block_sync();    // the second product of row block i-1 is over: its stage can be refilled
             if (lane == 0 && i > 0 && nload < nrb) fetch();
             __syncwarp();
         }
@@ -256,6 +266,7 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
         const unsigned bar_off = smem_u32(&xbar[0]) - smem_u32(&xch[0][0][0]);    // same offset in every block
         auto send = [&](long long j) {
             const int b = (int)(j & 3), xs = (int)(j & (XBUF - 1));
+            if (!mbar_wait(&pbar[b], (unsigned)((j >> 2) & 1), timed_out ? 64 : WAIT_LIMIT)) timed_out = true;
             float s = sh_part[b][xq][xr] + sh_part[b][xq + 4][xr];
             s += __shfl_xor_sync(0xffffffffu, s, 8);
             s += __shfl_xor_sync(0xffffffffu, s, 16);
@@ -265,13 +276,10 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
             if (xq < C) peer_store(peer_lo + word, s, peer_lo + bar);
             if (xq + 4 < C) peer_store(peer_hi + word, s, peer_hi + bar);
         };
-        __syncthreads();        // the first three first products are done
-        if (nrb > 0) send(0);
-        if (nrb > 1) send(1);
-        for (long long i = 0; i < nrb; ++i) {
-            __syncthreads();    // partial dots of row block i+2 are in place
-            if (i + 2 < nrb) send(i + 2);
-        }
+        // The send warp runs free of the block barrier: it follows the compute warps through pbar alone.  (A row
+        // block's buffer in sh_part is rewritten four row blocks later, which the compute warps reach only after
+        // the receive of a later row block, i.e. after this warp's later sends.)
+        for (long long j = 0; j < nrb; ++j) send(j);
     } else if (warp == WARPS + 1) {
         // ================= the receive warp =================
         const int xr = lane & 7, xq = lane >> 3;
@@ -305,10 +313,10 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
             }
         };
 
-        __syncthreads();
         if (nrb > 0) receive(0);
+        block_sync();
         for (long long i = 0; i < nrb; ++i) {
-            __syncthreads();    // the second product of row block i-1 is over: sh_u[(i+1) % 2] is free
+            block_sync();    // the second product of row block i-1 is over: sh_u[(i+1) % 2] is free
             if (i + 1 < nrb) receive(i + 1);
         }
     } else {
@@ -335,7 +343,7 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
         const unsigned unit1 = ((lm & 1) << 1) | (lm >> 1), unit2 = lm;
 
         // first product of the row block in `slot`; lanes t = 0 leave row g's partial dot product in dst[g]
-        auto first_product = [&](int slot, float *dst) {
+        auto first_product = [&](int slot, float *dst, uint64_t *ready) {
             const unsigned stage = ring + slot * STAGE_BYTES + lane_base;
             float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -346,6 +354,8 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
                 else mma_k16(e0, a, wf[ks][0], wf[ks][1]);
             }
             if (t == 0) dst[g] = (e0[0] + e1[0]) + (e0[3] + e1[3]);     // D[g][0] + D[g+8][1]
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ready);      // this warp's 8 partial dots are in place
         };
         // this unit's gradient: tile j of the second product is D[16 columns][n], n = 0, 1, 2 the three terms of u;
         // lane (g, t) holds columns 16 j + g (acc[j][0..1]) and 16 j + 8 + g (acc[j][2..3]) at n = 2t, 2t + 1
@@ -353,29 +363,29 @@ k_map_cluster(const __grid_constant__ ClusterParams p) {
 #pragma unroll
         for (int j = 0; j < NBLK / 2; ++j) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
 
-        // The pipeline: F = first product, S = send, R = receive, G = second product.  Iteration i runs S(i+2),
-        // R(i+1), F(i+3) and G(i) behind ONE block barrier; a row block's exchange has two iterations to land.
+        // The pipeline: F = first product, S = send, R = receive, G = second product.  Iteration i runs F(i+2),
+        // then S(i+2) as soon as all warps' partial dots are in (an mbarrier, no block barrier), R(i+1) and G(i),
+        // behind ONE block barrier: three stages hold data, three are in flight.
         int slot1 = 0;          // stage of the next first product
         unsigned round1 = 0;
         long long nfirst = 0;
         auto first_next = [&]() {
             if (nfirst >= nrb) return;
             if (!mbar_wait(&full[slot1], round1 & 1u, timed_out ? 64 : WAIT_LIMIT)) timed_out = true;
-            first_product(slot1, sh_part[nfirst & 3][warp]);
+            first_product(slot1, sh_part[nfirst & 3][warp], &pbar[nfirst & 3]);
             ++nfirst;
             if (++slot1 == STAGES) { slot1 = 0; ++round1; }
         };
         first_next();
         first_next();
-        first_next();
-        __syncthreads();
+        block_sync();
 
         Cursor cur;             // the row block of the second product
         cur.start(p, u0);
         int slot2 = 0;
         for (long long i = 0; i < nrb; ++i) {
-            __syncthreads();    // partial dots of row block i+2 and u of row block i are in place; G(i-1) is over
-            first_next();       // F(i+3)
+            block_sync();    // u of row block i is in place; G(i-1) is over everywhere
+            first_next();       // F(i+2)
 
             // ---- second product G(i): the transposed slab [256 columns x 8 rows] times (hi, mid, lo) [8 rows x 3]
             {
