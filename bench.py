@@ -44,6 +44,25 @@ NCU_TRAFFIC = {
 }
 
 
+# The same for one k_map_cluster launch of the cfg5 workload at full size
+# (profiles/k_map_cluster_cfg5.md).
+NCU_TRAFFIC_MAP = {
+    "sources_sha256": "405b136816127426e83e75c4f81579a7d29a5e3bd31ccc47d4b44866779f1613",
+    "workload": "cfg5", "map_kernel_bytes": 2819317000.0 + 7197184.0,
+}
+
+
+def measured_map_traffic(w):
+    import hashlib
+
+    h = hashlib.sha256()
+    for f in ("ccdc_map_cluster.cu", "ccdc_map.cu", "ccdc_internal.h"):
+        h.update((ROOT / "paper_1805_01993_b200" / "csrc" / f).read_bytes())
+    if h.hexdigest() != NCU_TRAFFIC_MAP["sources_sha256"] or w.name != NCU_TRAFFIC_MAP["workload"]:
+        return None
+    return NCU_TRAFFIC_MAP["map_kernel_bytes"]
+
+
 def measured_traffic(w):
     import hashlib
 
@@ -390,7 +409,7 @@ def run_ours(args, w):
     others = {n: {"achieved": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9,
                   "frac": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / peak, "ms_per_launch": stage_ms[n]}
               for n in stage_ms if n != top}
-    traffic = measured_traffic(w) if top == "k_decode_reduce" else None
+    traffic = measured_traffic(w) if top == "k_decode_reduce" else (measured_map_traffic(w) if top == "k_map" else None)
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
