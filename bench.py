@@ -47,7 +47,7 @@ NCU_TRAFFIC = {
 # The same for one k_map_cluster launch of the cfg5 workload at full size
 # (profiles/k_map_cluster_cfg5.md).
 NCU_TRAFFIC_MAP = {
-    "sources_sha256": "405b136816127426e83e75c4f81579a7d29a5e3bd31ccc47d4b44866779f1613",
+    "sources_sha256": "e6d191bdf680246c5cd9be6266b0062cf3fa2edeea9a32cb3752ae70637c1527",
     "workload": "cfg5", "map_kernel_bytes": 2819317000.0 + 7197184.0,
 }
 
@@ -56,7 +56,7 @@ def measured_map_traffic(w):
     import hashlib
 
     h = hashlib.sha256()
-    for f in ("ccdc_map_cluster.cu", "ccdc_map.cu", "ccdc_internal.h"):
+    for f in ("ccdc_map_cluster.cu", "ccdc_map_cluster.h", "ccdc_internal.h"):
         h.update((ROOT / "paper_1805_01993_b200" / "csrc" / f).read_bytes())
     if h.hexdigest() != NCU_TRAFFIC_MAP["sources_sha256"] or w.name != NCU_TRAFFIC_MAP["workload"]:
         return None

@@ -311,6 +311,16 @@ k_map(const __grid_constant__ MapParams p) {
     }
 }
 
+// Build-time choice of the Map kernel.  Measured on B200, K = 8 workload (336 files
+// of 8 MiB): loads through registers 0.68 ms; TMA with per-warp pipelines 0.88 ms
+// at 3 stages (1.2-1.5 ms at 4-6), TMA with block-wide stages 1.13 ms.  Both TMA
+// forms read X from DRAM once as well; what they lose is time per small box
+// (16 rows x 128 bytes).  Default: registers.
+#ifndef CCDC_MAP_USE_TMA
+#define CCDC_MAP_USE_TMA 0
+#endif
+
+#if CCDC_MAP_USE_TMA
 // ======================================================================
 // The same Map with X staged by the Tensor Memory Accelerator.
 // (opt-in: -DCCDC_MAP_USE_TMA=1)
@@ -571,14 +581,6 @@ k_map_tma(const __grid_constant__ MapTmaParams P) {
     if (timed_out) atomicExch(p.status, 1);
 }
 
-// Build-time choice of the Map kernel.  Measured on B200, K = 8 workload (336 files
-// of 8 MiB): loads through registers 0.68 ms; TMA with per-warp pipelines 0.88 ms
-// at 3 stages (1.2-1.5 ms at 4-6), TMA with block-wide stages 1.13 ms.  Both TMA
-// forms read X from DRAM once as well; what they lose is time per small box
-// (16 rows x 128 bytes).  Default: registers.
-#ifndef CCDC_MAP_USE_TMA
-#define CCDC_MAP_USE_TMA 0
-#endif
 
 // cuTensorMapEncodeTiled, fetched from the driver through the runtime (the
 // library does not link libcuda); nullptr if this driver does not offer it
@@ -596,6 +598,7 @@ encode_tiled_fn encode_tiled() {
     }();
     return fn;
 }
+#endif  // CCDC_MAP_USE_TMA
 
 const char *last_kernel = "";       // which kernel the last ccdc_map launched (reported, not synchronised)
 
