@@ -305,6 +305,20 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
                       void *const *dev_part, void *dev_coded, void *dev_out, void *dev_workspace,
                       void *stream);
 
+/* A whole linear-regression job from HOST memory (Section III: Map phase, Shuffle
+ * phase, Reduce outputs): copies node k's files host_x[k] ([files][rows][d] bf16),
+ * host_y[k] ([files][rows] fp32) and host_w ([d] bf16) into the device staging
+ * buffers dev_x[k], dev_y[k], dev_w, then ccdc_map into dev_part, ccdc_shuffle,
+ * and one device-to-host copy of the outputs into host_out (ccdc_out_bytes).
+ * All device buffers are the caller's, of the sizes the separate calls take
+ * (map_workspace: ccdc_map_workspace_bytes; dev_workspace: ccdc_workspace_bytes).
+ * Pinned host memory makes the copies asynchronous.  Enqueues on `stream` and
+ * returns without waiting; errors as ccdc_map and ccdc_shuffle. */
+int ccdc_job_host(ccdc_plan_t *plan, const void *const *host_x, const void *const *host_y, const void *host_w,
+                  long long rows, void *host_out, void *const *dev_x, void *const *dev_y, void *dev_w,
+                  void *const *dev_part, void *dev_coded, void *dev_out, void *map_workspace, void *dev_workspace,
+                  void *stream);
+
 /* Allocation-free variant of ccdc_decode_reduce (the paper has no counterpart:
  * this is a property of the library, not a step of the scheme).
  *

@@ -70,6 +70,7 @@ SIGNATURES = {
     "ccdc_decode_reduce_static": (_I, [_P, _PP, _P, _P, _P]),
     "ccdc_compression_shuffle": (_I, [_P, _PP, _PP, _P, _P]),
     "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
+    "ccdc_job_host": (_I, [_P, _PP, _PP, _P, _LL, _P, _PP, _PP, _P, _PP, _P, _P, _P, _P, _P]),
     "ccdc_strerror": (ctypes.c_char_p, [_I]),
     "ccdc_last_cuda_error": (_I, []),
     "ccdc_num_kernel_launches": (_I, []),
@@ -324,6 +325,15 @@ class Plan:
     def compression_shuffle(self, part, recv, out, stream=None):
         _check(lib().ccdc_compression_shuffle(self._h, _ptr_array(part), _ptr_array(recv), out.data_ptr(),
                                               _stream_handle(stream)), "ccdc_compression_shuffle")
+
+    def job_host(self, host_x, host_y, host_w, rows, host_out, dev_x, dev_y, dev_w, part, coded, out, map_workspace,
+                 workspace=None, stream=None):
+        """Map + shuffle from host tensors (pinned for asynchronous copies) through device staging buffers."""
+        _check(lib().ccdc_job_host(self._h, _ptr_array(host_x), _ptr_array(host_y), host_w.data_ptr(), rows,
+                                   host_out.data_ptr(), _ptr_array(dev_x), _ptr_array(dev_y), dev_w.data_ptr(),
+                                   _ptr_array(part), coded.data_ptr(), out.data_ptr(), map_workspace.data_ptr(),
+                                   workspace.data_ptr() if workspace is not None and workspace.numel() else None,
+                                   _stream_handle(stream)), "ccdc_job_host")
 
     def shuffle_host(self, host_part, host_out, part, coded, out, workspace=None, stream=None):
         """``host_part`` / ``host_out``: CPU tensors (pinned for asynchronous copies)."""

@@ -738,4 +738,32 @@ int ccdc_map_status(const ccdc_plan_t *plan, long long rows, const void *workspa
     return word == 0 ? CCDC_OK : CCDC_ESTATE;
 }
 
+int ccdc_job_host(ccdc_plan_t *plan, const void *const *host_x, const void *const *host_y, const void *host_w,
+                  long long rows, void *host_out, void *const *dev_x, void *const *dev_y, void *dev_w,
+                  void *const *dev_part, void *dev_coded, void *dev_out, void *map_workspace, void *dev_workspace,
+                  void *stream) {
+    if (!plan || !host_x || !host_y || !host_w || !host_out || !dev_x || !dev_y || !dev_w) return CCDC_EINVAL;
+    if (rows <= 0) return CCDC_ESIZE;
+    const ccdc_plan_s &P = *plan;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long d = P.row_elems;
+    for (int k = 0; k < P.K; ++k) {
+        if (!(P.nlocal[k] > 0 && ccdc_plan_node_is_local(plan, k))) continue;
+        if (!host_x[k] || !host_y[k] || !dev_x[k] || !dev_y[k]) return CCDC_EINVAL;
+        const size_t nrows = (size_t)P.node_nfiles[k] * (size_t)rows;
+        cudaError_t e = cudaMemcpyAsync(dev_x[k], host_x[k], nrows * (size_t)d * 2, cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dev_y[k], host_y[k], nrows * 4, cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+    }
+    cudaError_t e = cudaMemcpyAsync(dev_w, host_w, (size_t)d * 2, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+    int rc = ccdc_map(plan, (const void *const *)dev_x, (const void *const *)dev_y, dev_w, rows, dev_part,
+                      map_workspace, stream);
+    if (rc != CCDC_OK) return rc;
+    rc = ccdc_shuffle(plan, (const void *const *)dev_part, dev_coded, dev_out, dev_workspace, stream);
+    if (rc != CCDC_OK) return rc;
+    e = cudaMemcpyAsync(host_out, dev_out, ccdc_out_bytes(plan), cudaMemcpyDeviceToHost, st);
+    return e == cudaSuccess ? CCDC_OK : ccdc_internal_cuda_fail((int)e);
+}
+
 }  // extern "C"

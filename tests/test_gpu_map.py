@@ -143,6 +143,42 @@ def test_map_cluster_shapes(ccdc, K, r, N, Q, B, rows):
     assert ccdc.map_last_kernel() == ("k_map_cluster" if d in (2048, 4096, 8192, 16384) else "k_map")
 
 
+def test_job_from_host_buffers(ccdc):
+    """ccdc_job_host (copies in, Map, shuffle, copy out) gives bit for bit what the separate calls give on
+    device-resident inputs, and its outputs match the oracle."""
+    K, r, N, Q, B, rows = 4, 2, 12, 4, 512, 64
+    d = Q * B
+    X, y, w = regression_files(N, rows, d, seed=21)
+    plan = ccdc.Plan(K, r, N, Q, B, "float32")
+    hx = [torch.from_numpy(bf16_bits(X[plan.node_files(k)]).view(np.int16)).pin_memory() for k in range(K)]
+    hy = [torch.from_numpy(np.ascontiguousarray(y[plan.node_files(k)])).pin_memory() for k in range(K)]
+    hw = torch.from_numpy(bf16_bits(w).view(np.int16)).pin_memory()
+    dx = [torch.empty_like(t, device="cuda") for t in hx]
+    dy = [torch.empty_like(t, device="cuda") for t in hy]
+    dw = torch.empty_like(hw, device="cuda")
+    part = plan.alloc_partitions()
+    coded, out, wsp = plan.alloc(plan.coded_bytes), plan.alloc(plan.out_bytes), plan.alloc(plan.workspace_bytes)
+    mws = torch.empty(plan.map_workspace_bytes(rows) // 4, dtype=torch.float32, device="cuda")
+    host_out = torch.empty(out.numel(), dtype=out.dtype).pin_memory()
+    plan.job_host(hx, hy, hw, rows, host_out, dx, dy, dw, part, coded, out, mws, wsp)
+    torch.cuda.synchronize()
+    plan.map_status(rows, mws)
+    # the separate calls on the device copies
+    part2 = plan.alloc_partitions()
+    out2, coded2 = plan.alloc(plan.out_bytes), plan.alloc(plan.coded_bytes)
+    plan.map([t.view(torch.bfloat16) for t in dx], dy, dw.view(torch.bfloat16), rows, part2, mws)
+    plan.shuffle(part2, coded2, out2, wsp)
+    torch.cuda.synchronize()
+    assert torch.equal(host_out, out2.cpu())
+    # and the oracle on the binary64 Map values
+    v = np.stack([map_linear_regression(X[n], w, y[n], Q) for n in range(N)])
+    o = Oracle(K, r, N, Q, B, "float32")
+    ref = o.run(v)
+    _, a64 = o.direct()
+    got = host_out.numpy().view(np.float32).reshape(Q, B).astype(np.float64)
+    assert np.all(np.abs(got - ref) <= 1e-5 * a64)
+
+
 TMA_VARIANT = r"""
 import sys
 sys.path.insert(0, sys.argv[1])
