@@ -47,7 +47,7 @@ NCU_TRAFFIC = {
 # The same for one k_map_cluster launch of the cfg5 workload at full size
 # (profiles/k_map_cluster_cfg5.md).
 NCU_TRAFFIC_MAP = {
-    "sources_sha256": "e6d191bdf680246c5cd9be6266b0062cf3fa2edeea9a32cb3752ae70637c1527",
+    "sources_sha256": "9073590833bf861f2e86e9a411ea136aa774a1544de16fa0ed8ea94ef90487c4",
     "workload": "cfg5", "map_kernel_bytes": 2819317000.0 + 7197184.0,
 }
 

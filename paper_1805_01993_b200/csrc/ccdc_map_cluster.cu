@@ -8,16 +8,16 @@
 // barrier that follows its last use.  For every row block:
 //   1. first product: each warp multiplies its 256 columns of the slab by w on
 //      the tensor cores (mma.sync m16n8k16, A by ldmatrix, w held in registers
-//      as B fragments); the 8 warps' partial dot products are added in warp
-//      order;
-//   2. a send warp hands the block's 8 partial dots to all blocks of the
-//      cluster through distributed shared memory (asynchronous remote stores
+//      as B fragments) and leaves 8 partial dot products in shared memory;
+//   2. a send warp adds the 8 warps' partials (a fixed tree) and hands the
+//      block's 8 partial dots to all blocks of the cluster through
+//      distributed shared memory (asynchronous remote stores
 //      that count their bytes on the receiver's mbarrier); a receive warp adds
 //      the C blocks' partials in a fixed order, subtracts y, and splits the
 //      residual u into three bf16 terms (u = hi + mid + lo);
-//   3. second product: each warp multiplies the three terms (A rows 0..2) by the
-//      transposed slab (ldmatrix.trans, mma.sync m16n8k8) and accumulates its
-//      256 gradient columns in registers.
+//   3. second product: each warp multiplies the transposed slab (A by
+//      ldmatrix.trans, mma.sync m16n8k8) by the three terms (columns 0..2 of B)
+//      and accumulates its 256 gradient columns in registers.
 // The loop is software pipelined behind one block barrier per row block: the
 // first product runs two row blocks ahead of the second, a row block's partial
 // dots are sent in the iteration that computes them and received in the next.
