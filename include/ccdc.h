@@ -278,7 +278,10 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
  * buffers, so no separate all-gather is needed; the ranks must still synchronise
  * (on the host, or with stream events) before any of them launches
  * ccdc_decode_reduce, because a kernel of one rank never waits for another
- * rank.  Needs one file per batch or r <= 4 operands (CCDC_ESIZE otherwise). */
+ * rank.  Needs one file per batch or r <= 4 operands (CCDC_ESIZE otherwise). 
+ * The launches of ccdc_encode_fused, ccdc_decode_reduce and ccdc_shuffle can be
+ * captured in a CUDA graph once the plan's tables are on the device (after
+ * ccdc_plan_upload or a first call): they enqueue kernels only. */
 int ccdc_encode_fused_peers(ccdc_plan_t *plan, const void *const *part, void *const *peer_coded, void *stream);
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out,
                  void *workspace, void *stream);

@@ -183,6 +183,40 @@ def test_cfg5_shuffle_shape(ccdc):
     assert plan.coded_bits == 3_064_320
 
 
+def test_shuffle_replayed_from_a_cuda_graph(ccdc):
+    """The two launches of ccdc_shuffle (plus the final pass of a split loop) captured in a CUDA graph and
+    replayed on new inputs give the oracle's coded packets and outputs: small jobs are launch-bound and
+    are meant to be run this way."""
+    K, r, N, Q, B, dtype = 10, 3, 480, 10, 96, "float32"          # the K = 10 structure, short values, split loop
+    plan = ccdc.Plan(K, r, N, Q, B, dtype)
+    assert plan.workspace_bytes > 0
+    part = plan.alloc_partitions()
+    coded, out, ws = plan.alloc(plan.coded_bytes), plan.alloc(plan.out_bytes), plan.alloc(plan.workspace_bytes)
+    v0 = values_numpy(N, Q, B, dtype, seed=31)
+    plan.fill_partitions(part, torch.from_numpy(v0).cuda())
+    plan.shuffle(part, coded, out, ws)                            # tables uploaded, attributes set
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            plan.shuffle(part, coded, out, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    s, sp = plan.segment_elems, plan.coded_row_elems
+    for seed in (32, 33):
+        v = values_numpy(N, Q, B, dtype, seed=seed)
+        plan.fill_partitions(part, torch.from_numpy(v).cuda())
+        coded.zero_(); out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        o = Oracle(K, r, N, Q, B, dtype)
+        o.load_values(v)
+        o.shuffle()
+        assert np.array_equal(bits(coded).reshape(-1, sp)[:, :s], o.coded().reshape(-1, s))
+        assert_outputs(out, o, dtype)
+
+
 def test_special_float_patterns_survive_coding(ccdc):
     """-0.0, infinities and NaN payloads are carried bit for bit when b = 1."""
     K, r, N, Q, B = 4, 2, 6, 4, 8
