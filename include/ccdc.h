@@ -264,7 +264,10 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
  *   fp32 outputs are too when the workspace size is 0, and otherwise differ
  *   from it only by the grouping of the per-batch terms.
  * ccdc_shuffle: both, in order, on `stream`.
- *   coded: ccdc_coded_bytes; out: ccdc_out_bytes. */
+ *   coded: ccdc_coded_bytes; out: ccdc_out_bytes.
+ * These calls (and ccdc_shuffle) enqueue kernels only, so they can be captured in
+ * a CUDA graph once the plan's tables are on the device (after ccdc_plan_upload
+ * or a first call). */
 int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, void *stream);
 int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *coded, void *out,
                        void *workspace, void *stream);
@@ -278,10 +281,7 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
  * buffers, so no separate all-gather is needed; the ranks must still synchronise
  * (on the host, or with stream events) before any of them launches
  * ccdc_decode_reduce, because a kernel of one rank never waits for another
- * rank.  Needs one file per batch or r <= 4 operands (CCDC_ESIZE otherwise). 
- * The launches of ccdc_encode_fused, ccdc_decode_reduce and ccdc_shuffle can be
- * captured in a CUDA graph once the plan's tables are on the device (after
- * ccdc_plan_upload or a first call): they enqueue kernels only. */
+ * rank.  Needs one file per batch or r <= 4 operands (CCDC_ESIZE otherwise). */
 int ccdc_encode_fused_peers(ccdc_plan_t *plan, const void *const *part, void *const *peer_coded, void *stream);
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out,
                  void *workspace, void *stream);
