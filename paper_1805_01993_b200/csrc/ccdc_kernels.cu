@@ -274,13 +274,16 @@ k_gather(const __grid_constant__ GatherParams p) {
 #ifndef CCDC_STATIC_GATHER_VECTORS
 #define CCDC_STATIC_GATHER_VECTORS 2
 #endif
+#ifndef CCDC_GATHER_WIDE_ROW
+#define CCDC_GATHER_WIDE_ROW (1 << 15)    // one-file rows of at least this many words get blocks of twice the threads
+#endif
 constexpr int STHREADS = CCDC_STATIC_GATHER_THREADS;
 constexpr int SUNROLL = CCDC_STATIC_GATHER_VECTORS;
 
-template <int VEC, bool F32, int RS, bool B1>
-__global__ void __launch_bounds__(STHREADS)
+template <int VEC, bool F32, int RS, bool B1, int NT>
+__global__ void __launch_bounds__(NT)
 k_gather_static(const __grid_constant__ GatherParams p) {
-    constexpr long long TILE = (long long)STHREADS * VEC * SUNROLL;
+    constexpr long long TILE = (long long)NT * VEC * SUNROLL;
     const long long item = blockIdx.x;
     const long long row = item / p.spans_per_row;
     const long long span = item - row * p.spans_per_row;
@@ -300,7 +303,7 @@ k_gather_static(const __grid_constant__ GatherParams p) {
         for (int a = 0; a < RS; ++a)
 #pragma unroll
             for (int u = 0; u < SUNROLL; ++u) {
-                const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+                const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
                 v[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + j) : zero_words<VEC>();
             }
         // the other files of each batch, ascending; the loads of FU files are issued together
@@ -313,7 +316,7 @@ k_gather_static(const __grid_constant__ GatherParams p) {
                 for (int a = 0; a < RS; ++a)
 #pragma unroll
                     for (int u = 0; u < SUNROLL; ++u) {
-                        const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+                        const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
                         w[x][a][u] = (f + x < p.b && j < end && j < E[a].vl)
                                          ? load_words<VEC>(src + E[a].off + (f + x) * p.file_stride + j)
                                          : zero_words<VEC>();
@@ -329,7 +332,7 @@ k_gather_static(const __grid_constant__ GatherParams p) {
         }
 #pragma unroll
         for (int u = 0; u < SUNROLL; ++u) {
-            const long long j = base + ((long long)u * STHREADS + threadIdx.x) * VEC;
+            const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
 #pragma unroll
             for (int a = 1; a < RS; ++a) xor_into<VEC>(v[0][u], v[a][u]);
             if (j < end) {
@@ -602,7 +605,10 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         constexpr bool F32 = decltype(f32)::value;
         const bool lean = !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
         if (npeers > 0 && !lean) return CCDC_ESIZE;         // peer stores exist in the lean kernel only
-        const long long tile = lean ? (long long)STHREADS * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
+        // long one-file rows (the gradient-sized workload): 512-thread blocks measured 2 % faster; short rows lose with them
+        const bool wide = lean && b == 1 && T.n_max >= (long long)CCDC_GATHER_WIDE_ROW;
+        const int sthreads = wide ? 2 * STHREADS : STHREADS;
+        const long long tile = lean ? (long long)sthreads * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 148 SMs x 16 blocks
         long long tiles = 32;
@@ -614,8 +620,9 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         if (lean) {
             auto go = [&](auto rs) {
                 constexpr int RS = decltype(rs)::value;
-                if (b == 1) k_gather_static<VEC, F32, RS, true><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
-                else k_gather_static<VEC, F32, RS, false><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
+                if (wide) k_gather_static<VEC, F32, RS, true, 2 * STHREADS><<<(unsigned)blocks, 2 * STHREADS, 0, st>>>(gp);
+                else if (b == 1) k_gather_static<VEC, F32, RS, true, STHREADS><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
+                else k_gather_static<VEC, F32, RS, false, STHREADS><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
             };
             switch (T.na) {
             case 1: go(std::integral_constant<int, 1>()); break;
