@@ -355,12 +355,15 @@ def run_ours(args, w):
     stage_ms = {name: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
     enc_ms, dec_ms = stage_ms["k_gather(encode)"], stage_ms["k_decode_reduce"]
     ms_per_step = max_over_ranks(elapsed_ms, world, dev) / args.steps
-    # Small jobs are launch-bound (a step is a handful of kernels of a few microseconds): replay the
+    # Small jobs, and the Map job with its short shuffle, are launch-bound (a step is a handful of kernels,
+    # most of a few microseconds): replay the
     # step's launches as ONE CUDA graph, which is how a caller would run such a job repeatedly.  The
     # stage times above stay those of the eager launches.
     launch_mode, eager_ms = "eager launches", ms_per_step
-    if flush is not None and world == 1:
+    if (flush is not None or w.map_rows) and world == 1:
         try:
+            torch.cuda.synchronize()
+            eager_out = out.clone()                 # the replays must reproduce the eager step bit for bit
             side = torch.cuda.Stream(device=dev)
             side.wait_stream(stream)
             graph = torch.cuda.CUDAGraph()
@@ -371,7 +374,8 @@ def run_ours(args, w):
             stream.wait_stream(side)
             g_ms = []
             for i in range(args.warmup + args.steps):
-                flush.zero_()
+                if flush is not None:
+                    flush.zero_()
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
                 graph.replay()
@@ -379,6 +383,8 @@ def run_ours(args, w):
                 torch.cuda.synchronize()
                 if i >= args.warmup:
                     g_ms.append(a.elapsed_time(b))
+            if not torch.equal(out, eager_out):
+                raise RuntimeError("graph replay and eager launches disagree")
             launches += len(g_ms) * (launches // max(args.steps, 1))
             ms_per_step, launch_mode = sum(g_ms) / len(g_ms), "one CUDA graph replay per step"
         except Exception as exc:            # capture refused: keep the eager number
