@@ -112,10 +112,13 @@ struct ccdc_plan_s {
     std::vector<ccdc_ref> red_terms;
     const ccdc_ref *d_red_terms = nullptr;
 
+    int sm_count = 148;       // SMs the launch shapes are sized for (the device's count once uploaded)
     int device = -1;          // device holding the table copies, -1 = none
     void *d_blob = nullptr;   // one allocation for all of them
 };
 
+// implemented in ccdc_plan.cpp: sizes the split of the fused decode again for a device with sm_count SMs
+void ccdc_internal_resplit(ccdc_plan_s *plan, int sm_count);
 // implemented in ccdc_kernels.cu
 void ccdc_internal_release_device(ccdc_plan_s *plan);
 int ccdc_internal_cuda_fail(int cuda_error);    // records the error for ccdc_last_cuda_error; returns CCDC_ECUDA

@@ -610,9 +610,9 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         const int sthreads = wide ? 2 * STHREADS : STHREADS;
         const long long tile = lean ? (long long)sthreads * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
-        // leave the grid short of 148 SMs x 16 blocks
+        // leave the grid short of 16 blocks per SM
         long long tiles = 32;
-        while (tiles > 1 && gp.nrows * ((T.n_max + tile * tiles - 1) / (tile * tiles)) < 148 * 16) tiles /= 2;
+        while (tiles > 1 && gp.nrows * ((T.n_max + tile * tiles - 1) / (tile * tiles)) < (long long)P.sm_count * 16) tiles /= 2;
         gp.span_elems = tile * tiles;
         gp.spans_per_row = (T.n_max + gp.span_elems - 1) / gp.span_elems;
         const long long blocks = gp.nrows * gp.spans_per_row;
@@ -678,6 +678,10 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     if (e != cudaSuccess) return cuda_fail(e);
     if (plan->device == dev) return CCDC_OK;
     if (plan->device != -1) return CCDC_ESTATE;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    ccdc_internal_resplit(plan, sms);       // launch shapes for this device's SM count
     struct Piece { const void *src; size_t bytes; const void **dst; };
     ccdc_gather_table *tabs[4] = {&plan->enc_fused, &plan->cmb, &plan->enc_pk, &plan->dec_pk};
     Piece pieces[11];

@@ -12,7 +12,6 @@
 //                              row vectors with byte permutes
 // Every node maps its own copy of a file with the same code and the same fixed
 // summation order, so the replicas are bit-identical (no floating-point atomics).
-#include <cuda.h>            // CUtensorMap and its enums; the encoder itself is looked up at run time
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -311,294 +310,6 @@ k_map(const __grid_constant__ MapParams p) {
     }
 }
 
-// Build-time choice of the Map kernel.  Measured on B200, K = 8 workload (336 files
-// of 8 MiB): loads through registers 0.68 ms; TMA with per-warp pipelines 0.88 ms
-// at 3 stages (1.2-1.5 ms at 4-6), TMA with block-wide stages 1.13 ms.  Both TMA
-// forms read X from DRAM once as well; what they lose is time per small box
-// (16 rows x 128 bytes).  Default: registers.
-#ifndef CCDC_MAP_USE_TMA
-#define CCDC_MAP_USE_TMA 0
-#endif
-
-#if CCDC_MAP_USE_TMA
-// ======================================================================
-// The same Map with X staged by the Tensor Memory Accelerator.
-// (opt-in: -DCCDC_MAP_USE_TMA=1)
-// The busiest unit of the register version above is the L1/TEX path its 16-byte
-// loads take.  Here 2-D tiled bulk copies (16 rows x 64 columns = 2 KiB boxes of
-// X) go straight into rings of shared-memory stages; the copies complete on an
-// mbarrier per stage and never touch L1 or registers.
-// The warps read their MMA fragments from shared memory (each warp instruction
-// reads 4 rows x 128 bytes: conflict free without swizzling).
-// Every warp runs its own pipeline: lane 0 issues the warp's box copies into the
-// warp's ring of stages, each stage completes on its own mbarrier, and a stage
-// is refilled only after a __syncwarp that follows its consumption: no block
-// barrier inside the loops.  The only waits are on the warp's own copies; they
-// are bounded like the ticket wait and report through the status word.
-#ifndef CCDC_MAP_TMA_STAGES
-#define CCDC_MAP_TMA_STAGES 3
-#endif
-constexpr int TMA_STAGES = CCDC_MAP_TMA_STAGES;
-constexpr int TMA_BOX_BYTES = 16 * 64 * 2;      // 16 rows x 64 bf16 columns
-constexpr int TMA_WAIT_LIMIT = 1 << 22;
-
-struct MapTmaParams {
-    MapParams m;
-    CUtensorMap tmap[CCDC_MAX_K];       // node k: X as [files * rows][d] bf16, box 16 x 64
-};
-
-__device__ __forceinline__ unsigned smem_u32(const void *ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, unsigned bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// bounded wait for a stage's copies; false if the bound was hit
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity) {
-    for (int i = 0; i < TMA_WAIT_LIMIT; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
-__device__ __forceinline__ void tma_load_box(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar,
-                                             uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
-
-__global__ void __launch_bounds__(MAP_THREADS, 2)
-k_map_tma(const __grid_constant__ MapTmaParams P) {
-    const MapParams &p = P.m;
-    extern __shared__ __align__(128) unsigned char sh_raw[];
-    // every warp owns a ring of TMA_STAGES boxes (2 KiB each) and their barriers
-    unsigned char *ring = sh_raw;
-    uint32_t *sh_w = reinterpret_cast<uint32_t *>(sh_raw + MAP_WARPS * TMA_STAGES * TMA_BOX_BYTES);   // d/2 words
-    uint32_t *sh_u = sh_w + p.d / 2;                                            // 3 * rows/2 words
-    __shared__ __align__(8) uint64_t full[MAP_WARPS][TMA_STAGES];
-    __shared__ float sh_part[MAP_WARPS][16];
-    __shared__ long long sh_ticket;
-
-    const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    const int g = lane / 4, t = lane % 4;
-    if (threadIdx.x == 0) {
-        for (int w = 0; w < MAP_WARPS; ++w)
-            for (int s = 0; s < TMA_STAGES; ++s) mbar_init(&full[w][s], 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    for (long long i = threadIdx.x; i < p.d / 8; i += MAP_THREADS)
-        reinterpret_cast<uint4 *>(sh_w)[i] = __ldg(reinterpret_cast<const uint4 *>(p.w) + i);
-
-    unsigned char *my_ring = ring + warp * TMA_STAGES * TMA_BOX_BYTES;
-    uint64_t *my_full = full[warp];
-    const uint64_t keep = l2_policy_keep(), drop = l2_policy_drop();
-    unsigned phase = 0;                         // bit s = parity of this warp's next completion of stage s
-    bool timed_out = false;
-
-    const long long n1 = p.rows / 16, n2 = (p.d + GRAD_COLS - 1) / GRAD_COLS, per = n1 + n2;
-    const long long total = (p.njobs + CCDC_MAP_LAG) * per;
-    for (;;) {
-        __syncthreads();                        // sh_ticket, sh_u and sh_part are free again
-        if (threadIdx.x == 0) sh_ticket = atomicAdd(p.ticket, 1);
-        __syncthreads();
-        const long long tk = sh_ticket;
-        if (tk >= total) break;
-        const long long step_id = tk / per, slot = tk - step_id * per;
-        const bool pass1 = slot < n1;
-        const long long job = pass1 ? step_id : step_id - CCDC_MAP_LAG;
-        if (job < 0 || job >= p.njobs) continue;
-        const int k = node_of_job(p, job);
-        const long long file = job - p.first_job[k];
-        const CUtensorMap *map = &P.tmap[k];
-
-        if (pass1) {
-            // ---- u = X w - y for 16 rows; warp w takes columns [w d/8, (w+1) d/8), 64 per step.
-            // MMA row m of set sigma holds half (m%2) of box row 8 sigma + (m < 8 ? m/2 : 4 + (m-8)/2)
-            const long long row0 = slot * 16;
-            const int y0 = (int)(file * p.rows + row0);
-            const int x0 = (int)(warp * (p.d / MAP_WARPS));
-            const int steps = (int)(p.d / MAP_WARPS / 64);
-            auto issue = [&](int s) {                           // lane 0 of the warp
-                const int stage = s % TMA_STAGES;
-                mbar_expect_tx(&my_full[stage], TMA_BOX_BYTES);
-                tma_load_box(my_ring + stage * TMA_BOX_BYTES, map, x0 + 64 * s, y0, &my_full[stage], keep);
-            };
-            if (lane == 0)
-                for (int s = 0; s < TMA_STAGES && s < steps; ++s) issue(s);
-            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-            for (int s = 0; s < steps; ++s) {
-                const int stage = s % TMA_STAGES;
-                if (!mbar_wait(&my_full[stage], (phase >> stage) & 1u)) timed_out = true;
-                phase ^= 1u << stage;
-                const unsigned char *src = my_ring + stage * TMA_BOX_BYTES + (g / 2) * 128 + 64 * (g & 1) + 16 * t;
-                uint4 wv = make_uint4(0u, 0u, 0u, 0u);
-                if (g < 2) wv = *reinterpret_cast<const uint4 *>(sh_w + (x0 + 64 * s + 32 * g + 8 * t) / 2);
-#pragma unroll
-                for (int sg = 0; sg < 2; ++sg) {
-                    const uint4 va = *reinterpret_cast<const uint4 *>(src + (8 * sg) * 128);
-                    const uint4 vb = *reinterpret_cast<const uint4 *>(src + (8 * sg + 4) * 128);
-                    mma_bf16(acc[sg], va.x, vb.x, va.y, vb.y, wv.x, wv.y);
-                    mma_bf16(acc[sg], va.z, vb.z, va.w, vb.w, wv.z, wv.w);
-                }
-                __syncwarp();                                   // every lane has consumed the stage
-                if (lane == 0 && s + TMA_STAGES < steps) issue(s + TMA_STAGES);
-            }
-#pragma unroll
-            for (int sg = 0; sg < 2; ++sg) {
-                float lo = (g & 1) ? acc[sg][1] : acc[sg][0];   // D[m][m%2] for m = g
-                float hi = (g & 1) ? acc[sg][3] : acc[sg][2];   // ... for m = g + 8
-                lo += __shfl_xor_sync(0xffffffffu, lo, 4);      // the other half of the same row
-                hi += __shfl_xor_sync(0xffffffffu, hi, 4);
-                if (t == 0 && (g & 1) == 0) {
-                    sh_part[warp][8 * sg + g / 2] = lo;
-                    sh_part[warp][8 * sg + 4 + g / 2] = hi;
-                }
-            }
-            __syncthreads();
-            if (threadIdx.x < 16) {
-                float sum = sh_part[0][threadIdx.x];
-                for (int wv = 1; wv < MAP_WARPS; ++wv) sum += sh_part[wv][threadIdx.x];    // fixed order
-                const long long r = row0 + threadIdx.x;
-                p.u[job * p.rows + r] = sum - p.y[k][file * p.rows + r];
-                __threadfence();
-            }
-            __syncthreads();
-            if (threadIdx.x == 0) atomicAdd(p.done + job, 1);
-        } else {
-            // ---- g = X^T u for 512 columns; warp w takes 64 of them, 16 rows per step
-            const long long col0 = (slot - n1) * GRAD_COLS;
-            const long long j0 = col0 + warp * 64;
-            const bool active = j0 < p.d;
-            const int y0 = (int)(file * p.rows);
-            const int steps = (int)(p.rows / 16);
-            auto issue = [&](int s) {                           // lane 0 of the warp
-                const int stage = s % TMA_STAGES;
-                mbar_expect_tx(&my_full[stage], TMA_BOX_BYTES);
-                tma_load_box(my_ring + stage * TMA_BOX_BYTES, map, (int)j0, y0 + 16 * s, &my_full[stage], drop);
-            };
-            // the copies do not depend on u: start them before waiting for pass 1 of this file
-            if (active && lane == 0)
-                for (int s = 0; s < TMA_STAGES && s < steps; ++s) issue(s);
-            if (threadIdx.x == 0) {
-                const volatile int *done = p.done + job;
-                int polls = 0;
-                while (*done < (int)n1) {
-                    if (++polls > WAIT_LIMIT) { atomicExch(p.status, 1); break; }
-                    __nanosleep(100);
-                }
-                __threadfence();
-            }
-            __syncthreads();
-            const long long half_rows = p.rows / 2;
-            for (long long i = threadIdx.x; i < half_rows; i += MAP_THREADS) {
-                const float2 v2 = __ldcg(reinterpret_cast<const float2 *>(p.u + job * p.rows) + i);
-                const float v[2] = {v2.x, v2.y};
-                uint16_t term[3][2];
-                for (int e = 0; e < 2; ++e) {
-                    float rest = v[e];
-                    for (int sidx = 0; sidx < 3; ++sidx) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(rest);
-                        term[sidx][e] = __bfloat16_as_ushort(h);
-                        rest = rest - __bfloat162float(h);
-                    }
-                }
-                for (int sidx = 0; sidx < 3; ++sidx)
-                    sh_u[sidx * half_rows + i] = (uint32_t)term[sidx][0] | ((uint32_t)term[sidx][1] << 16);
-            }
-            __syncthreads();
-            if (active) {
-                float acc[8][4];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) acc[e][0] = acc[e][1] = acc[e][2] = acc[e][3] = 0.f;
-                for (int s = 0; s < steps; ++s) {
-                    const int stage = s % TMA_STAGES;
-                    if (!mbar_wait(&my_full[stage], (phase >> stage) & 1u)) timed_out = true;
-                    phase ^= 1u << stage;
-                    const unsigned char *tile = my_ring + stage * TMA_BOX_BYTES + 16 * g;
-                    const uint4 v0 = *reinterpret_cast<const uint4 *>(tile + (2 * t) * 128);
-                    const uint4 v1 = *reinterpret_cast<const uint4 *>(tile + (2 * t + 1) * 128);
-                    const uint4 v2 = *reinterpret_cast<const uint4 *>(tile + (2 * t + 8) * 128);
-                    const uint4 v3 = *reinterpret_cast<const uint4 *>(tile + (2 * t + 9) * 128);
-                    const long long r0 = 16LL * s + 2 * t;
-                    uint32_t a0 = 0u, a2 = 0u;
-                    if (g < 3) {
-                        a0 = sh_u[g * half_rows + r0 / 2];
-                        a2 = sh_u[g * half_rows + (r0 + 8) / 2];
-                    }
-                    const uint32_t w0[4] = {v0.x, v0.y, v0.z, v0.w}, w1[4] = {v1.x, v1.y, v1.z, v1.w};
-                    const uint32_t w2[4] = {v2.x, v2.y, v2.z, v2.w}, w3[4] = {v3.x, v3.y, v3.z, v3.w};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const uint32_t sel = (e & 1) ? 0x7632u : 0x5410u;
-                        const uint32_t b0 = __byte_perm(w0[e / 2], w1[e / 2], sel);
-                        const uint32_t b1 = __byte_perm(w2[e / 2], w3[e / 2], sel);
-                        mma_bf16(acc[e], a0, 0u, a2, 0u, b0, b1);
-                    }
-                    __syncwarp();                               // every lane has consumed the stage
-                    if (lane == 0 && s + TMA_STAGES < steps) issue(s + TMA_STAGES);
-                }
-                uint32_t *out = p.part[k] + file * p.d;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        const float hi = acc[e][c];
-                        const float mid = __shfl_down_sync(0xffffffffu, hi, 4);
-                        const float lo = __shfl_down_sync(0xffffffffu, hi, 8);
-                        acc[e][c] = (hi + mid) + lo;
-                    }
-                }
-                if (g == 0) {
-#pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        float4 lo4 = make_float4(acc[0][c], acc[1][c], acc[2][c], acc[3][c]);
-                        float4 hi4 = make_float4(acc[4][c], acc[5][c], acc[6][c], acc[7][c]);
-                        float *dst = reinterpret_cast<float *>(out) + j0 + 8 * (2 * t + c);
-                        *reinterpret_cast<float4 *>(dst) = lo4;
-                        *reinterpret_cast<float4 *>(dst + 4) = hi4;
-                    }
-                }
-            }
-        }
-    }
-    if (timed_out) atomicExch(p.status, 1);
-}
-
-
-// cuTensorMapEncodeTiled, fetched from the driver through the runtime (the
-// library does not link libcuda); nullptr if this driver does not offer it
-using encode_tiled_fn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                     const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                     CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-encode_tiled_fn encode_tiled() {
-    static encode_tiled_fn fn = [] {
-        void *ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            ptr = nullptr;
-        return reinterpret_cast<encode_tiled_fn>(ptr);
-    }();
-    return fn;
-}
-#endif  // CCDC_MAP_USE_TMA
 
 const char *last_kernel = "";       // which kernel the last ccdc_map launched (reported, not synchronised)
 
@@ -614,9 +325,9 @@ size_t residual_bytes(long long jobs, long long rows) { return ((size_t)(jobs * 
 size_t control_bytes(long long jobs) { return ((size_t)(jobs + 2) * 4 + 255) / 256 * 256; }
 
 // Which kernel maps a shape: the cluster kernel (X read once, staged by TMA) where it fits, unless
-// the library was built with -DCCDC_MAP_USE_CLUSTER=0 or with the per-warp TMA variant.
+// the library was built with -DCCDC_MAP_USE_CLUSTER=0.
 #ifndef CCDC_MAP_USE_CLUSTER
-#define CCDC_MAP_USE_CLUSTER (!CCDC_MAP_USE_TMA)
+#define CCDC_MAP_USE_CLUSTER 1
 #endif
 size_t pieces_bytes(long long jobs, long long rows, long long d) {
     return CCDC_MAP_USE_CLUSTER ? ccdc_map_cluster_pieces_bytes(jobs, rows, d) : 0;
@@ -677,40 +388,7 @@ int ccdc_map(ccdc_plan_t *plan, const void *const *files_x, const void *const *f
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
 
-#if CCDC_MAP_USE_TMA
-    // X staged by TMA: one tensor map per node ([files * rows][d] bf16, boxes of 16 rows x 64 columns)
-    if (encode_tiled()) {
-        static_assert(sizeof(MapTmaParams) < 32 * 1024, "kernel parameters");
-        MapTmaParams tp;
-        std::memset(&tp, 0, sizeof(tp));
-        tp.m = mp;
-        bool ok = true;
-        for (int k = 0; k < P.K && ok; ++k) {
-            if (P.node_nfiles[k] == 0) continue;
-            const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)(P.node_nfiles[k] * rows)};
-            const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
-            const cuuint32_t box[2] = {64, 16}, estr[2] = {1, 1};
-            ok = encode_tiled()(&tp.tmap[k], CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(files_x[k]), dims,
-                                strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-        }
-        if (ok) {
-            const size_t smem = (size_t)MAP_WARPS * TMA_STAGES * TMA_BOX_BYTES + (size_t)d * 2 + (size_t)rows * 6;
-            e = cudaFuncSetAttribute(k_map_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_map_tma, MAP_THREADS, smem);
-            if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
-            if (per_sm >= 1) {
-                per_sm = std::min(per_sm, CCDC_MAP_BLOCKS_PER_SM);
-                last_kernel = "k_map_tma";
-                k_map_tma<<<(unsigned)(sms * per_sm), MAP_THREADS, smem, st>>>(tp);
-                ccdc_internal_count_launch();
-                e = cudaGetLastError();
-                return e == cudaSuccess ? CCDC_OK : ccdc_internal_cuda_fail((int)e);
-            }
-        }
-    }
-#endif
-    // loads through registers (also the fallback when the tensor-map encoder is unavailable)
+    // loads through registers
     const size_t smem = (size_t)d * 2 + (size_t)rows * 6;
     if (smem > 32 * 1024) {
         e = cudaFuncSetAttribute(k_map, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

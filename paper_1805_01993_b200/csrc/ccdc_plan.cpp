@@ -88,14 +88,15 @@ int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
 }
 
 // split of the batch loop of the fused decode over `nout` output rows: enough
-// thread blocks to fill the GPU (148 SMs x 8 resident blocks) while a block
-// still walks a fair number of batches
+// thread blocks to fill the GPU (SMs x 8 resident blocks) while a block
+// still walks a fair number of batches.  P.sm_count is 148 (B200) until the
+// tables are uploaded, when the device's own count replaces it.
 void choose_split(ccdc_plan_s &P, long long nout) {
     auto split_for = [&](int threads, long long &per_chunk, int &nchunk) {
         const long long tile = (long long)threads * P.vec * CCDC_DECODE_VECTORS;
         const long long tiles_per_seg = (P.s + tile - 1) / tile;
         const long long base = std::max(1LL, nout * P.r * tiles_per_seg);
-        const long long want = (148LL * 8 + base - 1) / base;
+        const long long want = ((long long)P.sm_count * 8 + base - 1) / base;
         const long long cap = std::max(1LL, P.nterm / 8);
         const long long nch = std::max(1LL, std::min(want, cap));
         per_chunk = (P.nterm + nch - 1) / nch;
@@ -111,7 +112,7 @@ void choose_split(ccdc_plan_s &P, long long nout) {
         P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS) {
         long long per_chunk = 0;
         int nchunk = 0;
-        if (split_for(CCDC_DECODE_THREADS_SHORT, per_chunk, nchunk) >= 148LL * 6) {
+        if (split_for(CCDC_DECODE_THREADS_SHORT, per_chunk, nchunk) >= (long long)P.sm_count * 6) {
             P.decode_threads = CCDC_DECODE_THREADS_SHORT;
             P.terms_per_chunk = per_chunk;
             P.nchunk = nchunk;
@@ -503,6 +504,13 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
 
 }  // namespace
 
+void ccdc_internal_resplit(ccdc_plan_s *plan, int sm_count) {
+    if (sm_count < 1 || sm_count == plan->sm_count) return;
+    plan->sm_count = sm_count;
+    if (plan->compression_mode) return;
+    choose_split(*plan, plan->shard_world > 1 ? (long long)plan->out_rows.size() : plan->J * plan->K);
+}
+
 extern "C" {
 
 int ccdc_plan_sharded(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, int jobs, int rank,
@@ -554,6 +562,9 @@ void ccdc_plan_destroy(ccdc_plan_t *plan) {
     ccdc_internal_release_device(plan);
     delete plan;
 }
+
+int ccdc_plan_decode_threads(const ccdc_plan_t *p) { return p && !p->compression_mode ? p->decode_threads : 0; }
+int ccdc_plan_decode_chunks(const ccdc_plan_t *p) { return p && !p->compression_mode ? p->nchunk : 0; }
 
 long long ccdc_plan_num_jobs(const ccdc_plan_t *p) { return p ? p->J : 0; }
 long long ccdc_plan_num_batches(const ccdc_plan_t *p) { return p ? p->nbatch : 0; }

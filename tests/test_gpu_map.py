@@ -179,25 +179,20 @@ def test_job_from_host_buffers(ccdc):
     assert np.all(np.abs(got - ref) <= 1e-5 * a64)
 
 
-TMA_VARIANT = r"""
+REGISTER_VARIANT = r"""
 import sys
 sys.path.insert(0, sys.argv[1])
 from pathlib import Path
 from paper_1805_01993_b200 import build, ccdc
-ccdc._LIB_PATH = build.build_variant(Path(sys.argv[2]) / "libccdc_tma.so", ("CCDC_MAP_USE_TMA=1",))
+ccdc._LIB_PATH = build.build_variant(Path(sys.argv[2]) / "libccdc_reg.so", ("CCDC_MAP_USE_CLUSTER=0",))
 sys.path.insert(0, str(Path(sys.argv[1]) / "tests"))
 import test_gpu_map as t
 t.run_job(ccdc, 4, 2, 12, 4, 128, rows=32, seed=7)
 t.run_job(ccdc, 4, 3, 8, 4, 512, rows=48, seed=8)
 t.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)
-print("tma variant ok")
+assert ccdc.map_last_kernel() == "k_map"
+print("register variant ok")
 """
-
-
-REGISTER_VARIANT = TMA_VARIANT.replace('"libccdc_tma.so", ("CCDC_MAP_USE_TMA=1",)', '"libccdc_reg.so", ("CCDC_MAP_USE_CLUSTER=0",)') \
-    .replace("t.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)",
-             't.run_job(ccdc, 8, 3, 112, 8, 1024, rows=128, seed=9)\nassert ccdc.map_last_kernel() == "k_map"') \
-    .replace("tma variant ok", "register variant ok")
 
 
 def test_register_kernel_on_cluster_shapes(ccdc, tmp_path):
@@ -214,21 +209,6 @@ def test_register_kernel_on_cluster_shapes(ccdc, tmp_path):
     res = subprocess.run([sys.executable, str(script), str(root), str(tmp_path)], capture_output=True, text=True,
                          timeout=900)
     assert res.returncode == 0 and "register variant ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
-
-
-def test_tma_variant_of_the_map(ccdc, tmp_path):
-    """The opt-in Map kernel that stages X with TMA bulk tensor copies and mbarriers is
-    built into a scratch directory and held to the same parity as the default."""
-    import subprocess
-    import sys
-    from pathlib import Path
-
-    root = Path(__file__).resolve().parent.parent
-    script = tmp_path / "tma_variant.py"
-    script.write_text(TMA_VARIANT)
-    res = subprocess.run([sys.executable, str(script), str(root), str(tmp_path)], capture_output=True, text=True,
-                         timeout=900)
-    assert res.returncode == 0 and "tma variant ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
 
 
 def test_map_refuses_bad_shapes(ccdc):
