@@ -34,44 +34,40 @@ from paper_1805_01993_b200.inputs import CONFIGS, DEFAULT_SEED, values_numpy, va
 METRIC = "shuffle GB/s (combine+encode+decode+reduce)"
 UNIT = "GB/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one k_decode_reduce
-# launch from the ncu capture summarised in profiles/k_decode_reduce_cfg4_B128000.md,
-# taken on the cfg4 structure with B = 128000; it grows in proportion to B.  Only
-# valid for the kernel sources it was measured on (hash below); otherwise null.
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel of a
+# workload, from the ncu captures summarised under profiles/ (file named per entry).  A capture taken
+# at a shorter value length is scaled by the value length (every byte the kernel moves grows in
+# proportion to it) and the line says "scaled".  An entry is only valid for the kernel sources it was
+# measured on (hash over the files listed); otherwise the line reports null.
 NCU_TRAFFIC = {
-    "sources_sha256": "b73c826ab66f29f54abeea7dd41991c71527af7cad34369b878fe90e4d7250e5",
-    "workload": "cfg4", "value_elems": 128000, "decode_kernel_bytes": 3527696000.0 + 10893312.0,
+    # workload: (kernel, sources sha256, value elements of the capture, DRAM bytes of that launch, profile)
+}
+TRAFFIC_SOURCES = {
+    "k_decode_reduce": ("ccdc_kernels.cu", "ccdc_internal.h", "ccdc_plan.cpp"),
+    "k_gather(encode)": ("ccdc_kernels.cu", "ccdc_internal.h", "ccdc_plan.cpp"),
+    "k_map": ("ccdc_map_cluster.cu", "ccdc_map_cluster.h", "ccdc_internal.h"),
 }
 
 
-# The same for one k_map_cluster launch of the cfg5 workload at full size
-# (profiles/k_map_cluster_cfg5.md).
-NCU_TRAFFIC_MAP = {
-    "sources_sha256": "9073590833bf861f2e86e9a411ea136aa774a1544de16fa0ed8ea94ef90487c4",
-    "workload": "cfg5", "map_kernel_bytes": 2819317000.0 + 7197184.0,
-}
-
-
-def measured_map_traffic(w):
+def sources_hash(kernel):
     import hashlib
 
     h = hashlib.sha256()
-    for f in ("ccdc_map_cluster.cu", "ccdc_map_cluster.h", "ccdc_internal.h"):
+    for f in TRAFFIC_SOURCES[kernel]:
         h.update((ROOT / "paper_1805_01993_b200" / "csrc" / f).read_bytes())
-    if h.hexdigest() != NCU_TRAFFIC_MAP["sources_sha256"] or w.name != NCU_TRAFFIC_MAP["workload"]:
-        return None
-    return NCU_TRAFFIC_MAP["map_kernel_bytes"]
+    return h.hexdigest()
 
 
-def measured_traffic(w):
-    import hashlib
-
-    h = hashlib.sha256()
-    for f in ("ccdc_kernels.cu", "ccdc_internal.h"):
-        h.update((ROOT / "paper_1805_01993_b200" / "csrc" / f).read_bytes())
-    if h.hexdigest() != NCU_TRAFFIC["sources_sha256"] or not w.name.startswith(NCU_TRAFFIC["workload"]):
-        return None
-    return NCU_TRAFFIC["decode_kernel_bytes"] * w.B / NCU_TRAFFIC["value_elems"]
+def measured_traffic(w, kernel):
+    """(DRAM bytes per launch of `kernel` on workload w, how they were obtained) or (None, None)."""
+    base = w.name.split("[")[0]
+    entry = NCU_TRAFFIC.get(base)
+    if not entry or entry[0] != kernel or sources_hash(kernel) != entry[1]:
+        return None, None
+    _, _, elems, dram_bytes, profile = entry
+    if elems == w.B:
+        return dram_bytes, f"ncu capture of this launch ({profile})"
+    return dram_bytes * w.B / elems, f"scaled by {w.B}/{elems} from an ncu capture at B={elems} ({profile})"
 
 
 # ---------------------------------------------------------------- byte counts
@@ -169,6 +165,27 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(power)}
 
 
+def host_cpu():
+    """model name and core counts of the host the oracle is timed on."""
+    model = "unknown"
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                model = line.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    try:
+        usable = len(os.sched_getaffinity(0))
+    except AttributeError:
+        usable = os.cpu_count()
+    return {"cpu_model": model, "host_cores": os.cpu_count(), "host_cores_usable": usable}
+
+
+SAMPLE_REASON = ("value length shortened so that the single-threaded oracle finishes in the seconds "
+                 "the benchmark allows; every step is element-wise along the value, so the rate does not depend on it")
+
+
 # ---------------------------------------------------------------- oracle legs
 def oracle_sample_shape(w, target_seconds):
     """Same K, r, N, Q with the value shortened so one oracle pass takes about
@@ -237,7 +254,8 @@ def run_reference(args, w):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic", "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "sample_reason": SAMPLE_REASON if B < w.B else "full size", **host_cpu()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }))
@@ -293,7 +311,10 @@ def run_ours(args, w):
         gen.manual_seed(rank_seed(rank))
         d = w.Q * w.B
         canon = torch.randn((w.N, w.map_rows, d), generator=gen, device=dev).to(torch.bfloat16)
-        ycan = torch.randn((w.N, w.map_rows), generator=gen, device=dev)
+        # y_n = X_n w* + 0.01 N(0,1), as the workload states (drawn on the device; one file at a time)
+        w_star = torch.randn(d, generator=gen, device=dev)
+        ycan = torch.stack([canon[n].float() @ w_star for n in range(w.N)])
+        ycan += 0.01 * torch.randn((w.N, w.map_rows), generator=gen, device=dev)
         files_x = [canon[plan.node_files(k)].contiguous() for k in range(w.K)]
         files_y = [ycan[plan.node_files(k)].contiguous() for k in range(w.K)]
         del canon, ycan
@@ -318,12 +339,19 @@ def run_ours(args, w):
                    "k_decode_reduce": by["decode_kernel"] // share,
                    "all_gather(coded rows)": by["coded_write"] * (world - 1) // max(world, 1)}
     input_bytes = sum(plan.partition_bytes(k) for k in range(w.K)) + map_bytes
-    # inputs that fit in L2 (126 MB) would be served from it on every repeat: flush between steps
+    # inputs that fit in L2 (126 MB) would be served from it on every repeat: between steps 512 MB are
+    # written, then another 512 MB are read; the read pass pushes the dirty lines the write leaves in L2
+    # out to memory, so that the step starts with a cold AND clean L2 instead of paying for their write-back
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if input_bytes < (1 << 30) else None
+    drain = torch.zeros(128 << 20, dtype=torch.int32, device=dev) if flush is not None else None
+
+    def flush_l2():
+        flush.zero_()
+        drain.sum()
 
     def one_step(events=None):
         if flush is not None:
-            flush.zero_()
+            flush_l2()
         for i, (_, fn) in enumerate(stages):
             if events is not None:
                 events[i].record(stream)
@@ -350,6 +378,8 @@ def run_ours(args, w):
     barrier()
     launches = ccdc.num_kernel_launches() - launches0
     clocks = sampler.stop() if rank == 0 else None
+    if w.map_rows:
+        plan.map_status(w.map_rows, map_ws)     # raises if a bounded wait inside the Map ran out: no number then
     # with a flush between steps the bracket would include it: sum the steps instead
     elapsed_ms = start.elapsed_time(end) if flush is None else sum(e[0].elapsed_time(e[-1]) for e in ev)
     stage_ms = {name: statistics.mean(e[i].elapsed_time(e[i + 1]) for e in ev) for i, (name, _) in enumerate(stages)}
@@ -375,7 +405,7 @@ def run_ours(args, w):
             g_ms = []
             for i in range(args.warmup + args.steps):
                 if flush is not None:
-                    flush.zero_()
+                    flush_l2()
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record(stream)
                 graph.replay()
@@ -385,8 +415,12 @@ def run_ours(args, w):
                     g_ms.append(a.elapsed_time(b))
             if not torch.equal(out, eager_out):
                 raise RuntimeError("graph replay and eager launches disagree")
+            if w.map_rows:
+                plan.map_status(w.map_rows, map_ws)
             launches += len(g_ms) * (launches // max(args.steps, 1))
             ms_per_step, launch_mode = sum(g_ms) / len(g_ms), "one CUDA graph replay per step"
+        except ccdc.CcdcError:
+            raise
         except Exception as exc:            # capture refused: keep the eager number
             launch_mode = f"eager launches (graph capture failed: {type(exc).__name__})"
     value = whole_job_value(1 if sharded else world, by["iv_read"], ms_per_step)
@@ -465,11 +499,16 @@ def run_ours(args, w):
         peak, peak_kind = 6650.0, "fallback"
     # the dominant kernel of the step (the exchange between GPUs is reported beside it, not as a kernel)
     top = max((n for n in stage_ms if not n.startswith("all_gather")), key=stage_ms.get)
-    achieved = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
+    NOMINAL = 8000.0                                    # GB/s, the B200's nominal HBM3e rate
+    algorithmic_gbs = stage_bytes[top] / (stage_ms[top] * 1e-3) / 1e9
     others = {n: {"achieved": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9,
-                  "frac": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / peak, "ms_per_launch": stage_ms[n]}
+                  "frac": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / peak,
+                  "frac_nominal": stage_bytes[n] / (stage_ms[n] * 1e-3) / 1e9 / NOMINAL, "ms_per_launch": stage_ms[n]}
               for n in stage_ms if n != top}
-    traffic = measured_traffic(w) if top == "k_decode_reduce" else (measured_map_traffic(w) if top == "k_map" else None)
+    traffic, traffic_kind = measured_traffic(w, top)
+    # with a DRAM byte count for this kernel the achieved rate is DRAM bytes over time (bytes served
+    # from L2 do not count as HBM traffic); the algorithmic rate stays beside it
+    achieved = (traffic if traffic else stage_bytes[top]) / (stage_ms[top] * 1e-3) / 1e9
 
     cpu = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -478,7 +517,8 @@ def run_ours(args, w):
         bs = sample_bytes(w, Bs)
         cpu = {"value": bs["iv_read"] / secs / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"{w.name} with B={Bs} of {w.B} elements per value (same K, r, N, Q), one pass, "
-                         f"{secs:.1f} s"}
+                         f"{secs:.1f} s",
+               "sample_reason": SAMPLE_REASON if Bs < w.B else "full size", **host_cpu()}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -488,16 +528,21 @@ def run_ours(args, w):
         "config": {"workload": w.name, "parallelism": f"nodes sharded over {world} GPUs, all-gather of coded rows" if sharded
                    else f"{world} independent job(s), one per GPU", "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
                    "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
-                          f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written between steps, steps timed one by one"),
+                          f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written, then 512 MB read, between steps; steps timed one by one"),
                    "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": plan.J,
                    "launch": launch_mode, **({"eager_ms_per_step": eager_ms} if launch_mode.startswith("one") else {}),
                    **({"map_kernel": ccdc.map_last_kernel()} if w.map_rows else {}),
                    "load_per_JQT": plan.coded_bits / (plan.J * w.Q * 32 * w.B),
                    "coded_bits": plan.coded_bits, "iv_bytes_per_step": by["iv_read"],
                    "algorithmic_bytes_per_step": by["total"] + map_bytes,
-                   "hbm_frac_whole_step": (by["total"] + map_bytes) / (ms_per_step * 1e-3) / 1e9 / peak},
+                   "hbm_frac_whole_step": (by["total"] + map_bytes) / (ms_per_step * 1e-3) / 1e9 / peak,
+                   "hbm_frac_whole_step_nominal": (by["total"] + map_bytes) / (ms_per_step * 1e-3) / 1e9 / NOMINAL},
         "roofline": {"bound": "hbm", "kernel": top, "achieved": achieved, "peak": peak,
-                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_nominal": achieved / NOMINAL, "nominal_peak": NOMINAL,
+                     "achieved_kind": "DRAM bytes (ncu) / time" if traffic else "algorithmic bytes / time",
+                     "algorithmic_gbs": algorithmic_gbs, "algorithmic_frac": algorithmic_gbs / peak,
+                     "algorithmic_bytes": stage_bytes[top], "traffic": traffic, "traffic_kind": traffic_kind,
                      "ms_per_launch": stage_ms[top], "other_kernels": others},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
     }

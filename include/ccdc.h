@@ -134,8 +134,25 @@ void ccdc_plan_destroy(ccdc_plan_t *plan);
 
 /* Copies the schedule tables to the current device (cudaMalloc + cudaMemcpy,
  * synchronous).  Optional: the first step call on a plan does it implicitly.
- * After it no step function allocates.  CCDC_ENOMEM / CCDC_ECUDA on failure. */
+ * After it no step function allocates.  CCDC_ENOMEM / CCDC_ECUDA on failure.
+ * The launch shapes of a plan are sized for 148 SMs (B200) when it is created;
+ * the upload sizes them again for the current device's SM count, which can
+ * change ccdc_workspace_bytes on another GPU model: query it after the upload
+ * there. */
 int  ccdc_plan_upload(ccdc_plan_t *plan);
+
+/* Launch shape of the fused decode (ccdc_decode_reduce), chosen by the planner:
+ * threads per block, and the number of blocks (chunks) the loop over a job's
+ * batches is split into (1 = no workspace needed).  ccdc_plan_tune_decode
+ * overrides the choice, e.g. from a timing sweep; it changes
+ * ccdc_workspace_bytes.  Allowed: chunks in 1..batches per job; threads 128 for
+ * plans with several files per batch, r <= 4 and an even segment length, else
+ * 512 or 1024 (CCDC_EINVAL otherwise); only before the tables are uploaded
+ * (CCDC_ESTATE after).  Results do not depend on the shape for int32; for fp32
+ * the grouping of the per-batch terms follows the chunks (Eq. (1) is a sum). */
+int  ccdc_plan_decode_threads(const ccdc_plan_t *plan);
+int  ccdc_plan_decode_chunks(const ccdc_plan_t *plan);
+int  ccdc_plan_tune_decode(ccdc_plan_t *plan, int threads, int chunks);
 
 /* ---------------------------------------------------------------- queries
  * All host side, valid for the plan's lifetime.  Index arguments out of range
@@ -258,11 +275,14 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
  * ccdc_decode_reduce: launch 2.  For node k, each of its output words: over
  *   the batches of the job in ascending order, the local pre-combined word, or
  *   the coded word XOR the r-1 cancellable pre-combined words (decoding of
- *   Section IV-B), accumulated as Eq. (1) demands.  workspace:
+ *   Section IV-B), accumulated as Eq. (1) demands.  When the loop over the
+ *   batches is split over several blocks, each leaves its partial sum in the
+ *   workspace and a second small launch adds them in chunk order.  workspace:
  *   ccdc_workspace_bytes (may be NULL if that is 0); it is fully overwritten
- *   before it is read.  int32 outputs are bit-identical to the stepwise path;
- *   fp32 outputs are too when the workspace size is 0, and otherwise differ
- *   from it only by the grouping of the per-batch terms.
+ *   before it is read.  int32 outputs are
+ *   bit-identical to the stepwise path; fp32 outputs are too when the
+ *   workspace size is 0, and otherwise differ from it only by the grouping of
+ *   the per-batch terms.
  * ccdc_shuffle: both, in order, on `stream`.
  *   coded: ccdc_coded_bytes; out: ccdc_out_bytes.
  * These calls (and ccdc_shuffle) enqueue kernels only, so they can be captured in
@@ -351,6 +371,12 @@ int ccdc_decode_reduce_static(ccdc_plan_t *plan, const void *const *part, const 
 const char *ccdc_strerror(int status);
 int ccdc_last_cuda_error(void);          /* cudaError_t of the last CCDC_ECUDA on this thread */
 int ccdc_num_kernel_launches(void);      /* kernels launched by this library so far (process wide) */
+/* Which kernel form the calling thread's most recent gather launch (ccdc_combine, ccdc_encode,
+ * ccdc_decode, ccdc_encode_fused, the first launch of ccdc_compression_shuffle) and most recent
+ * ccdc_decode_reduce used, e.g. "k_gather_static<vec=4,operands=2,files=1,vectors=2,threads=512>";
+ * "" before the first.  Static per-thread strings. */
+const char *ccdc_last_gather_kernel(void);
+const char *ccdc_last_decode_kernel(void);
 
 #ifdef __cplusplus
 }

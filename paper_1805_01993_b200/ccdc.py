@@ -34,6 +34,9 @@ SIGNATURES = {
     "ccdc_coded_send_bytes": (_SZ, [_P]),
     "ccdc_plan_destroy": (None, [_P]),
     "ccdc_plan_upload": (_I, [_P]),
+    "ccdc_plan_decode_threads": (_I, [_P]),
+    "ccdc_plan_decode_chunks": (_I, [_P]),
+    "ccdc_plan_tune_decode": (_I, [_P, _I, _I]),
     "ccdc_plan_num_jobs": (_LL, [_P]),
     "ccdc_plan_num_batches": (_LL, [_P]),
     "ccdc_plan_num_groups": (_LL, [_P]),
@@ -74,6 +77,8 @@ SIGNATURES = {
     "ccdc_strerror": (ctypes.c_char_p, [_I]),
     "ccdc_last_cuda_error": (_I, []),
     "ccdc_num_kernel_launches": (_I, []),
+    "ccdc_last_gather_kernel": (ctypes.c_char_p, []),
+    "ccdc_last_decode_kernel": (ctypes.c_char_p, []),
 }
 
 
@@ -193,6 +198,18 @@ class Plan:
 
     def coded_row_position(self, g, a):
         return lib().ccdc_plan_coded_row_position(self._h, g, a)
+
+    @property
+    def decode_threads(self):
+        return lib().ccdc_plan_decode_threads(self._h)
+
+    @property
+    def decode_chunks(self):
+        return lib().ccdc_plan_decode_chunks(self._h)
+
+    def tune_decode(self, threads, chunks):
+        """fixes the launch shape of the fused decode (before the tables are uploaded)."""
+        _check(lib().ccdc_plan_tune_decode(self._h, threads, chunks), "ccdc_plan_tune_decode")
 
     @property
     def coded_send_bytes(self):
@@ -355,6 +372,16 @@ class Plan:
 
 def num_kernel_launches() -> int:
     return lib().ccdc_num_kernel_launches()
+
+
+def last_gather_kernel() -> str:
+    """Kernel form of this thread's most recent gather launch (combine, encode, decode, fused encode)."""
+    return lib().ccdc_last_gather_kernel().decode()
+
+
+def last_decode_kernel() -> str:
+    """Kernel form of this thread's most recent fused decode launch."""
+    return lib().ccdc_last_decode_kernel().decode()
 
 
 def map_last_kernel() -> str:

@@ -15,6 +15,15 @@
 #ifndef CCDC_DECODE_THREADS_SHORT
 #define CCDC_DECODE_THREADS_SHORT 1024  // used instead when one such block covers a whole segment
 #endif
+#ifndef CCDC_DECODE_THREADS_FILES
+#define CCDC_DECODE_THREADS_FILES 128   // used when several files of a batch are loaded together
+#endif
+#ifndef CCDC_DECODE_FILES_MAX
+#define CCDC_DECODE_FILES_MAX 4         // most files of a batch loaded together (4, 2; 1 = batch-by-batch kernel)
+#endif
+#ifndef CCDC_DECODE_GROUP_WORDS
+#define CCDC_DECODE_GROUP_WORDS 40      // most words per thread a batch may keep in flight
+#endif
 #ifndef CCDC_DECODE_VECTORS
 #define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
@@ -59,6 +68,7 @@ struct ccdc_gather_table {
     int na = 0;
     long long n_max = 0;            // largest row length
     bool uniform = true;            // no row carries its own file count (nf = 0 everywhere)
+    long long nf_max = 0;           // largest per-row file count (tables that are not uniform)
     // device copies
     const ccdc_row *d_rows = nullptr;
     const ccdc_ref *d_refs = nullptr;
@@ -85,6 +95,8 @@ struct ccdc_plan_s {
     int vec = 1;              // widest vector (words) dividing s and len: 4, 2 or 1
     int term_stride = 0;      // refs per term of the fused decode: 1 + max(r-1, 1)
     int decode_threads = CCDC_DECODE_THREADS;   // block size of the fused decode
+    int decode_files = 1;     // files of a batch whose loads the fused decode issues together
+    bool tuned = false;       // the caller fixed the decode's launch shape (ccdc_plan_tune_decode)
     int nchunk = 1;           // split of the batch loop in the fused decode
     long long terms_per_chunk = 0;
 

@@ -22,9 +22,11 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstdio>
 #include <algorithm>
 #include <cstring>
 #include <type_traits>
+#include <utility>
 
 #include "ccdc_internal.h"
 
@@ -38,11 +40,51 @@ constexpr int GUNROLL = CCDC_GATHER_VECTORS;
 constexpr int STAGES = CCDC_GATHER_STAGES;
 
 thread_local int g_last_cuda_error = 0;
+thread_local char g_last_gather[96] = "";     // the instantiations this thread launched last
+thread_local char g_last_decode[96] = "";
 std::atomic<int> g_launches{0};
 
 int cuda_fail(cudaError_t e) {
     g_last_cuda_error = (int)e;
     return CCDC_ECUDA;
+}
+
+// ------------------------------------------- programmatic dependent launch
+// Every kernel here is launched so that the GPU may schedule its blocks while
+// the previous kernel of the stream is still draining: it first lets its own
+// dependent go (pdl_trigger), reads what no kernel writes (the plan's tables),
+// and calls pdl_wait -- which returns once the previous kernel has finished and
+// its writes are visible -- before it touches any data buffer.  Nothing is read
+// or written before the wait except plan tables, so the order of the stream is
+// kept exactly; what is saved is the launch latency between short kernels.
+// (A hardware dependency of the launch, not a spin: there is nothing to time out.)
+#ifndef CCDC_USE_PDL
+#define CCDC_USE_PDL 1
+#endif
+__device__ __forceinline__ void pdl_trigger() {
+#if CCDC_USE_PDL
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
+}
+__device__ __forceinline__ void pdl_wait() {
+#if CCDC_USE_PDL
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+#endif
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), long long grid, int block, size_t smem, cudaStream_t st, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = CCDC_USE_PDL ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 // ---------------------------------------------------------------- vectors
@@ -198,8 +240,10 @@ k_gather(const __grid_constant__ GatherParams p) {
     const long long begin = span * p.span_elems;
     const long long end = min(R.n, begin + p.span_elems);
     if (begin >= end) return;
+    pdl_trigger();
     if (threadIdx.x < p.na) sh_refs[threadIdx.x] = p.refs[row * p.na + threadIdx.x];
     __syncthreads();
+    pdl_wait();
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[R.dst_node] + R.dst_off;
     const int a0 = R.coded_off >= 0 ? -1 : 0;
@@ -265,25 +309,28 @@ k_gather(const __grid_constant__ GatherParams p) {
 }
 
 // Lean variant for the common shapes: RS operands known at compile time, no
-// coded input, every row summing the plan's b files.  The RS x SUNROLL loads
-// of a file step are issued from registers before they are consumed; no shared
-// memory, no barrier.
+// coded input.  The loads of G files of every operand (RS x G x SU vectors) are
+// issued from registers before any is consumed; no shared memory, no barrier.
+// A batch of more than G files takes further groups of G, added in file order.
 #ifndef CCDC_STATIC_GATHER_THREADS
 #define CCDC_STATIC_GATHER_THREADS 256
-#endif
-#ifndef CCDC_STATIC_GATHER_VECTORS
-#define CCDC_STATIC_GATHER_VECTORS 2
 #endif
 #ifndef CCDC_GATHER_WIDE_ROW
 #define CCDC_GATHER_WIDE_ROW (1 << 15)    // one-file rows of at least this many words get blocks of twice the threads
 #endif
+#ifndef CCDC_GATHER_FILES_VECTORS
+#define CCDC_GATHER_FILES_VECTORS 2       // vectors per thread per tile when several files are loaded together
+#endif
+#ifndef CCDC_GATHER_GROUP_WORDS
+#define CCDC_GATHER_GROUP_WORDS 48        // most words per thread a group of files may keep in flight
+#endif
 constexpr int STHREADS = CCDC_STATIC_GATHER_THREADS;
-constexpr int SUNROLL = CCDC_STATIC_GATHER_VECTORS;
+constexpr int FSU = CCDC_GATHER_FILES_VECTORS;
 
-template <int VEC, bool F32, int RS, bool B1, int NT>
+template <int VEC, bool F32, int RS, int G, int SU, int NT>
 __global__ void __launch_bounds__(NT)
 k_gather_static(const __grid_constant__ GatherParams p) {
-    constexpr long long TILE = (long long)NT * VEC * SUNROLL;
+    constexpr long long TILE = (long long)NT * VEC * SU;
     const long long item = blockIdx.x;
     const long long row = item / p.spans_per_row;
     const long long span = item - row * p.spans_per_row;
@@ -292,46 +339,43 @@ k_gather_static(const __grid_constant__ GatherParams p) {
     const long long begin = span * p.span_elems;
     const long long end = min(R.n, begin + p.span_elems);
     if (begin >= end) return;
+    pdl_trigger();
     ccdc_ref E[RS];
 #pragma unroll
     for (int a = 0; a < RS; ++a) E[a] = p.refs[row * RS + a];
+    pdl_wait();
+    const int nb = G == 1 ? 1 : (R.nf > 0 ? (int)R.nf : p.b);      // files summed per operand
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[p.replicas > 0 ? 0 : R.dst_node] + R.dst_off + p.dst_add;
     for (long long base = begin; base < end; base += TILE) {
-        Words<VEC> v[RS][SUNROLL];
+        Words<VEC> v[RS][SU];
+        for (int f0 = 0; f0 < nb; f0 += G) {
+            Words<VEC> w[G][RS][SU];
 #pragma unroll
-        for (int a = 0; a < RS; ++a)
-#pragma unroll
-            for (int u = 0; u < SUNROLL; ++u) {
-                const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
-                v[a][u] = (j < end && j < E[a].vl) ? load_words<VEC>(src + E[a].off + j) : zero_words<VEC>();
-            }
-        // the other files of each batch, ascending; the loads of FU files are issued together
-        constexpr int FU = RS * SUNROLL >= 6 ? 2 : (RS * SUNROLL >= 3 ? 4 : 8);
-        for (int f = 1; !B1 && f < p.b; f += FU) {
-            Words<VEC> w[FU][RS][SUNROLL];
-#pragma unroll
-            for (int x = 0; x < FU; ++x)
+            for (int x = 0; x < G; ++x)
 #pragma unroll
                 for (int a = 0; a < RS; ++a)
 #pragma unroll
-                    for (int u = 0; u < SUNROLL; ++u) {
+                    for (int u = 0; u < SU; ++u) {
                         const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
-                        w[x][a][u] = (f + x < p.b && j < end && j < E[a].vl)
-                                         ? load_words<VEC>(src + E[a].off + (f + x) * p.file_stride + j)
+                        w[x][a][u] = (f0 + x < nb && j < end && j < E[a].vl)
+                                         ? load_words<VEC>(src + E[a].off + (f0 + x) * p.file_stride + j)
                                          : zero_words<VEC>();
                     }
 #pragma unroll
-            for (int x = 0; x < FU; ++x)
-                if (f + x < p.b) {
+            for (int x = 0; x < G; ++x) {
+                if (f0 + x >= nb) break;
 #pragma unroll
-                    for (int a = 0; a < RS; ++a)
+                for (int a = 0; a < RS; ++a)
 #pragma unroll
-                        for (int u = 0; u < SUNROLL; ++u) add_into<VEC, F32>(v[a][u], w[x][a][u]);
-                }
+                    for (int u = 0; u < SU; ++u) {
+                        if (f0 + x == 0) v[a][u] = w[0][a][u];              // the sum starts from the first file's value
+                        else add_into<VEC, F32>(v[a][u], w[x][a][u]);
+                    }
+            }
         }
 #pragma unroll
-        for (int u = 0; u < SUNROLL; ++u) {
+        for (int u = 0; u < SU; ++u) {
             const long long j = base + ((long long)u * NT + threadIdx.x) * VEC;
 #pragma unroll
             for (int a = 1; a < RS; ++a) xor_into<VEC>(v[0][u], v[a][u]);
@@ -352,11 +396,17 @@ k_gather_static(const __grid_constant__ GatherParams p) {
 // value if k stores the batch, else the coded word XOR the r-1 cancellable
 // pre-combined words (Section IV-B decoding), added to the accumulator
 // (Eq. (1)).  Decoded packets never reach memory.
+//
+// When the batch loop is split over several blocks (chunks), every block
+// leaves its partial sum in the workspace and k_sum_chunks adds them in chunk
+// order.  (Letting the block that finishes a cell last add them inside this
+// kernel was tried: no faster on any workload, and the extra code disturbed
+// the register allocation of the streaming loop.)
 struct DecodeParams {
     const uint32_t *part[CCDC_MAX_K];
     const uint32_t *coded;
-    uint32_t *out;          // [out rows][len] when nchunk == 1
-    uint32_t *ws;           // [nchunk][out rows][len] otherwise
+    uint32_t *out;          // [out rows][len]
+    uint32_t *ws;           // [nchunk][out rows][len] when nchunk > 1
     const ccdc_ref *terms;  // [out rows][r][nterm][TS]
     const int *out_rows;    // the out rows to compute (node-sharded plans), or NULL for all
     long long nlist;        // how many
@@ -364,23 +414,40 @@ struct DecodeParams {
     long long len, s;
     long long file_stride;
     long long tiles_per_seg;
+    long long tile_span;    // consecutive tiles of a segment one block walks
+    long long spans_per_seg;
     long long nterm, terms_per_chunk;
     int K, r, b, TS, nchunk;
     int stage_terms;        // terms staged in shared memory at a time
 };
 
-// R1S >= 0: r-1 = R1S is a compile-time constant, so a batch's loads are issued
-// together; with one file per batch (B1) the loads of DEPTH consecutive batches
-// are issued before any is consumed (about 64 KiB of loads in flight per SM is
-// what the HBM read rate needs).  R1S < 0: any r, batch by batch.
-template <int VEC, bool F32, int NT, int R1S, bool B1>
-__global__ void __launch_bounds__(NT)
+// R1S >= 0: r-1 = R1S is a compile-time constant and the loads of a batch --
+// the coded word and G files of each of the r-1 operands, or G files of a
+// local batch -- are issued together; batches of more than G files take
+// further groups of G.  The loads of DEPTH consecutive batches are issued
+// before any is consumed (about 64 KiB of loads in flight per SM is what the
+// HBM read rate needs).  R1S < 0: any r, batch by batch.
+// A block walks `tile_span` consecutive tiles of its segment; when its whole chunk of the term table
+// fits the shared-memory stage it is staged once for all of them.
+// Blocks per SM the register allocation is held to (the compiler's own choice moves with every
+// change to the kernel, and the streaming rate follows the resident threads): blocks of 512 threads
+// with little in flight per thread at 3 per SM (40 registers), with more at 2 (64); several files in
+// flight: up to 80 registers.
+constexpr int decode_min_blocks(int vec, int nt, int r1s, int g) {
+    if (g > 1) return nt <= 128 ? 6 : nt <= 256 ? 3 : 2;
+    if (nt >= 1024) return 1;
+    if (r1s < 0) return vec <= 2 ? 3 : 2;
+    return (1 + r1s) * vec * CCDC_DECODE_DEPTH <= 16 ? 3 : 2;
+}
+
+template <int VEC, bool F32, int NT, int R1S, int G>
+__global__ void __launch_bounds__(NT, decode_min_blocks(VEC, NT, R1S, G))
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
     constexpr long long TILE = (long long)NT * VEC * DUNROLL;
     extern __shared__ ccdc_ref sh_terms[];
 
     long long item = blockIdx.x;
-    const long long tile = item % p.tiles_per_seg; item /= p.tiles_per_seg;
+    const long long span = item % p.spans_per_seg; item /= p.spans_per_seg;
     const int i = (int)(item % p.r); item /= p.r;
     const int chunk = (int)(item % p.nchunk);
     const long long li = item / p.nchunk;
@@ -388,36 +455,47 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
     const long long orow = p.out_rows ? p.out_rows[li] : li;
 
     const long long seglen = min(p.s, max(0LL, p.len - (long long)i * p.s));
-    if (tile * TILE >= seglen) return;
     const int k = (int)(orow % p.K);
     const uint32_t *src = p.part[k];
-    const long long j0 = tile * TILE + (long long)threadIdx.x * VEC;
     const int r1 = p.r - 1;
 
     const long long t_begin = (long long)chunk * p.terms_per_chunk;
     const long long t_end = min(p.nterm, t_begin + p.terms_per_chunk);
     const ccdc_ref *table = p.terms + ((orow * p.r + i) * p.nterm) * p.TS;
+    // one-file batches: a block takes a single tile (SPAN false: no loop state in the streaming loop)
+    constexpr bool SPAN = G > 1;
+    const bool staged_once = SPAN && t_end - t_begin <= p.stage_terms;
+    pdl_trigger();
+    if (staged_once) {
+        for (int x = threadIdx.x; x < (int)(t_end - t_begin) * p.TS; x += NT) sh_terms[x] = table[t_begin * p.TS + x];
+        __syncthreads();
+    }
+    pdl_wait();
 
+    const long long tile_first = SPAN ? span * p.tile_span : span;
+    const long long tile_end = SPAN ? min(p.tiles_per_seg, (span + 1) * p.tile_span) : span + 1;
+    for (long long tile = tile_first; tile < tile_end; ++tile) {
+    if (tile * TILE >= seglen) break;
+    const long long j0 = tile * TILE + (long long)threadIdx.x * VEC;
     Words<VEC> acc[DUNROLL];
 #pragma unroll
     for (int u = 0; u < DUNROLL; ++u) acc[u] = zero_words<VEC>();
 
     for (long long t0 = t_begin; t0 < t_end; t0 += p.stage_terms) {
         const int nt = (int)min((long long)p.stage_terms, t_end - t0);
-        __syncthreads();
-        for (int x = threadIdx.x; x < nt * p.TS; x += NT) sh_terms[x] = table[t0 * p.TS + x];
-        __syncthreads();
+        if (!staged_once) {
+            __syncthreads();
+            for (int x = threadIdx.x; x < nt * p.TS; x += NT) sh_terms[x] = table[t0 * p.TS + x];
+            __syncthreads();
+        }
         if constexpr (R1S >= 0) {
-            constexpr int DEPTH = B1 ? CCDC_DECODE_DEPTH : 1;
-            // one operand: a single word vector, or the batch sum over its b files
-            auto fetch = [&](long long off, long long j, long long vl) -> Words<VEC> {
-                if (B1) return j < vl ? load_words<VEC>(src + off + j) : zero_words<VEC>();
-                return batch_sum<VEC, F32>(src, off, j, vl, p.b, p.file_stride);
-            };
+            constexpr int NSLOT = (1 + R1S * G) > G ? (1 + R1S * G) : G;     // vectors a batch keeps in flight
+            constexpr int DEPTH = NSLOT * VEC * DUNROLL <= 18 ? CCDC_DECODE_DEPTH : 1;
+            const int nb = G == 1 ? 1 : p.b;
             for (int t = 0; t < nt; t += DEPTH) {
-                Words<VEC> v[DEPTH][1 + R1S][DUNROLL];
+                Words<VEC> v[DEPTH][NSLOT][DUNROLL];
 #pragma unroll
-                for (int x = 0; x < DEPTH; ++x) {              // every load of DEPTH batches first
+                for (int x = 0; x < DEPTH; ++x) {              // every first-group load of DEPTH batches first
                     if (t + x >= nt) break;
                     const ccdc_ref *e = sh_terms + (t + x) * p.TS;
                     const long long coded_off = e[0].off;
@@ -425,25 +503,58 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                     for (int u = 0; u < DUNROLL; ++u) {
                         const long long j = j0 + (long long)u * NT * VEC;
                         if (coded_off < 0) {
-                            v[x][0][u] = fetch(e[1].off, j, seglen);
+                            const uint32_t *q = src + e[1].off + j;
+#pragma unroll
+                            for (int f = 0; f < G; ++f)
+                                v[x][f][u] = (f < nb && j < seglen) ? load_words<VEC>(q + f * p.file_stride) : zero_words<VEC>();
                         } else {
                             v[x][0][u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
 #pragma unroll
-                            for (int c = 1; c <= R1S; ++c)
-                                v[x][c][u] = fetch(e[c].off, j, min(seglen, e[c].vl));
+                            for (int c = 1; c <= R1S; ++c) {
+                                const uint32_t *q = src + e[c].off + j;
+                                const bool ok = j < seglen && j < e[c].vl;
+#pragma unroll
+                                for (int f = 0; f < G; ++f)
+                                    v[x][1 + (c - 1) * G + f][u] = (f < nb && ok) ? load_words<VEC>(q + f * p.file_stride)
+                                                                                  : zero_words<VEC>();
+                            }
                         }
                     }
                 }
 #pragma unroll
                 for (int x = 0; x < DEPTH; ++x) {              // then consume them in batch order
                     if (t + x >= nt) break;
-                    const bool local = sh_terms[(t + x) * p.TS].off < 0;
+                    const ccdc_ref *e = sh_terms + (t + x) * p.TS;
+                    const bool local = e[0].off < 0;
 #pragma unroll
                     for (int u = 0; u < DUNROLL; ++u) {
-                        Words<VEC> val = v[x][0][u];
-                        if (!local) {
+                        const long long j = j0 + (long long)u * NT * VEC;
+                        // sum over the files of one operand whose first group sits in slots first..first+G-1
+                        auto operand = [&](int first, const ccdc_ref E, long long vl) -> Words<VEC> {
+                            Words<VEC> sum = v[x][first][u];
 #pragma unroll
-                            for (int c = 1; c <= R1S; ++c) xor_into<VEC>(val, v[x][c][u]);
+                            for (int f = 1; f < G; ++f)
+                                if (f < nb) add_into<VEC, F32>(sum, v[x][first + f][u]);
+                            for (int f0 = G; f0 < nb; f0 += G) {            // batches of more than G files
+                                Words<VEC> w[G];
+#pragma unroll
+                                for (int f = 0; f < G; ++f)
+                                    w[f] = (f0 + f < nb && j < vl) ? load_words<VEC>(src + E.off + j + (f0 + f) * p.file_stride)
+                                                                   : zero_words<VEC>();
+#pragma unroll
+                                for (int f = 0; f < G; ++f)
+                                    if (f0 + f < nb) add_into<VEC, F32>(sum, w[f]);
+                            }
+                            return sum;
+                        };
+                        Words<VEC> val;
+                        if (local) {
+                            val = operand(0, e[1], seglen);
+                        } else {
+                            val = v[x][0][u];
+#pragma unroll
+                            for (int c = 1; c <= R1S; ++c)
+                                xor_into<VEC>(val, operand(1 + (c - 1) * G, e[c], min(seglen, e[c].vl)));
                         }
                         add_into<VEC, F32>(acc[u], val);
                     }
@@ -456,20 +567,20 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                 Words<VEC> v[DUNROLL];
                 if (coded_off < 0) {
                     const ccdc_ref E = e[1];
-    #pragma unroll
+#pragma unroll
                     for (int u = 0; u < DUNROLL; ++u) {
                         const long long j = j0 + (long long)u * NT * VEC;
                         v[u] = batch_sum<VEC, F32>(src, E.off, j, seglen, p.b, p.file_stride);
                     }
                 } else {
-    #pragma unroll
+#pragma unroll
                     for (int u = 0; u < DUNROLL; ++u) {
                         const long long j = j0 + (long long)u * NT * VEC;
                         v[u] = j < seglen ? load_words<VEC>(p.coded + coded_off + j) : zero_words<VEC>();
                     }
                     for (int c = 1; c <= r1; ++c) {
                         const ccdc_ref E = e[c];
-    #pragma unroll
+#pragma unroll
                         for (int u = 0; u < DUNROLL; ++u) {
                             const long long j = j0 + (long long)u * NT * VEC;
                             if (j < seglen)
@@ -477,22 +588,24 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
                         }
                     }
                 }
-    #pragma unroll
+#pragma unroll
                 for (int u = 0; u < DUNROLL; ++u) add_into<VEC, F32>(acc[u], v[u]);
             }
-    
         }
     }
-    uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) +
-                    orow * p.len + (long long)i * p.s;
+    const long long cell_off = orow * p.len + (long long)i * p.s;
+    // the output, or this chunk's partial sum when the batch loop is split
+    uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) + cell_off;
 #pragma unroll
     for (int u = 0; u < DUNROLL; ++u) {
         const long long j = j0 + (long long)u * NT * VEC;
         if (j < seglen) store_words<VEC>(dst + j, acc[u]);
     }
+    }   // tiles of the span
 }
 
-// final pass of the split batch loop: out = ((ws[0] + ws[1]) + ...) in chunk order
+// final pass of a split batch loop when the decode kernel leaves the partial sums in the workspace:
+// out = ((ws[0] + ws[1]) + ...) in chunk order
 template <bool F32>
 __global__ void __launch_bounds__(DTHREADS)
 k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, const int *__restrict__ out_rows,
@@ -501,6 +614,8 @@ k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, const 
     if (x >= nlist * len) return;
     const long long li = x / len;
     const long long e = (out_rows ? out_rows[li] : li) * len + (x - li * len);
+    pdl_trigger();
+    pdl_wait();
     uint32_t acc = ws[e];
     for (int c = 1; c < nchunk; ++c) acc = add_word<F32>(acc, ws[(long long)c * n + e]);
     out[e] = acc;
@@ -529,13 +644,23 @@ k_reduce(const __grid_constant__ ReduceParams p) {
     if (j >= p.len) return;
     const int k = (int)(orow % p.K);
     const ccdc_ref *terms = p.terms + orow * p.nterm;
+    pdl_trigger();
+    pdl_wait();
     Words<VEC> acc = zero_words<VEC>();
-    for (long long t = 0; t < p.nterm; ++t) {
-        const ccdc_ref E = terms[t];
-        Words<VEC> v = E.vl <= 0 ? batch_sum<VEC, F32>(p.part[k], E.off, j, p.len, E.vl < 0 ? (int)-E.vl : p.b,
-                                                       p.file_stride)
-                                 : load_words<VEC>(p.decoded[k] + E.off + j);
-        add_into<VEC, F32>(acc, v);
+    for (long long t = 0; t < p.nterm; t += 4) {            // four batches' loads in flight, added in batch order
+        Words<VEC> v[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            if (t + x >= p.nterm) break;
+            const ccdc_ref E = terms[t + x];
+            v[x] = E.vl <= 0 ? batch_sum<VEC, F32>(p.part[k], E.off, j, p.len, E.vl < 0 ? (int)-E.vl : p.b, p.file_stride)
+                             : load_words<VEC>(p.decoded[k] + E.off + j);
+        }
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            if (t + x >= p.nterm) break;
+            add_into<VEC, F32>(acc, v[x]);
+        }
     }
     store_words<VEC>(p.out + orow * p.len + j, acc);
 }
@@ -603,12 +728,18 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
     return dispatch(P, [&](auto vec, auto f32) -> int {
         constexpr int VEC = decltype(vec)::value;
         constexpr bool F32 = decltype(f32)::value;
-        const bool lean = !coded_in && T.uniform && T.na >= 1 && T.na <= 4;
+        const bool lean = !coded_in && T.na >= 1 && T.na <= 4;
         if (npeers > 0 && !lean) return CCDC_ESIZE;         // peer stores exist in the lean kernel only
+        const long long bmax = T.uniform ? b : T.nf_max;    // most files summed per operand
+        // files whose loads are issued together: all of a small batch, fewer while the registers
+        // of a thread would have to hold more than 48 words of them
+        int group = bmax <= 1 ? 1 : bmax == 2 ? 2 : 4;
+        while (group > 2 && T.na * group * VEC * FSU > CCDC_GATHER_GROUP_WORDS) group /= 2;
         // long one-file rows (the gradient-sized workload): 512-thread blocks measured 2 % faster; short rows lose with them
-        const bool wide = lean && b == 1 && T.n_max >= (long long)CCDC_GATHER_WIDE_ROW;
+        const bool wide = lean && group == 1 && T.n_max >= (long long)CCDC_GATHER_WIDE_ROW;
         const int sthreads = wide ? 2 * STHREADS : STHREADS;
-        const long long tile = lean ? (long long)sthreads * VEC * SUNROLL : (long long)GTHREADS * VEC * GUNROLL;
+        const int svectors = group == 1 ? 2 : FSU;          // vectors per thread per tile
+        const long long tile = lean ? (long long)sthreads * VEC * svectors : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
         // leave the grid short of 16 blocks per SM
         long long tiles = 32;
@@ -620,9 +751,10 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         if (lean) {
             auto go = [&](auto rs) {
                 constexpr int RS = decltype(rs)::value;
-                if (wide) k_gather_static<VEC, F32, RS, true, 2 * STHREADS><<<(unsigned)blocks, 2 * STHREADS, 0, st>>>(gp);
-                else if (b == 1) k_gather_static<VEC, F32, RS, true, STHREADS><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
-                else k_gather_static<VEC, F32, RS, false, STHREADS><<<(unsigned)blocks, STHREADS, 0, st>>>(gp);
+                if (wide) launch_kernel(k_gather_static<VEC, F32, RS, 1, 2, 2 * STHREADS>, blocks, 2 * STHREADS, 0, st, gp);
+                else if (group == 1) launch_kernel(k_gather_static<VEC, F32, RS, 1, 2, STHREADS>, blocks, STHREADS, 0, st, gp);
+                else if (group == 2) launch_kernel(k_gather_static<VEC, F32, RS, 2, FSU, STHREADS>, blocks, STHREADS, 0, st, gp);
+                else launch_kernel(k_gather_static<VEC, F32, RS, 4, FSU, STHREADS>, blocks, STHREADS, 0, st, gp);
             };
             switch (T.na) {
             case 1: go(std::integral_constant<int, 1>()); break;
@@ -630,12 +762,15 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
             case 3: go(std::integral_constant<int, 3>()); break;
             default: go(std::integral_constant<int, 4>()); break;
             }
+            std::snprintf(g_last_gather, sizeof(g_last_gather), "k_gather_static<vec=%d,operands=%d,files=%d,vectors=%d,threads=%d>",
+                          VEC, T.na, group, svectors, sthreads);
             return check_launch();
         }
         const size_t smem = slots_bytes(VEC);
         int rc = allow_shared_memory(k_gather<VEC, F32>, smem);
         if (rc != CCDC_OK) return rc;
-        k_gather<VEC, F32><<<(unsigned)blocks, GTHREADS, smem, st>>>(gp);
+        launch_kernel(k_gather<VEC, F32>, blocks, GTHREADS, smem, st, gp);
+        std::snprintf(g_last_gather, sizeof(g_last_gather), "k_gather<vec=%d,threads=%d>", VEC, GTHREADS);
         return check_launch();
     });
 }
@@ -669,6 +804,8 @@ void ccdc_internal_release_device(ccdc_plan_s *plan) {
 extern "C" {
 
 int ccdc_last_cuda_error(void) { return g_last_cuda_error; }
+const char *ccdc_last_gather_kernel(void) { return g_last_gather; }
+const char *ccdc_last_decode_kernel(void) { return g_last_decode; }
 int ccdc_num_kernel_launches(void) { return g_launches.load(); }
 
 int ccdc_plan_upload(ccdc_plan_t *plan) {
@@ -775,7 +912,7 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
         rp.tiles_per_row = (P.len + tile - 1) / tile;
         const long long blocks = rp.nout * rp.tiles_per_row;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
-        k_reduce<VEC, F32><<<(unsigned)blocks, DTHREADS, 0, st>>>(rp);
+        launch_kernel(k_reduce<VEC, F32>, blocks, DTHREADS, 0, st, rp);
         return check_launch();
     });
 }
@@ -834,38 +971,55 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         constexpr bool F32 = decltype(f32)::value;
         const long long tile = (long long)P.decode_threads * VEC * DUNROLL;
         dp.tiles_per_seg = (P.s + tile - 1) / tile;
-        const long long blocks = dp.nlist * P.nchunk * P.r * dp.tiles_per_seg;
+        // a block walks several tiles of its segment while the grid keeps 16 blocks per SM (amortises
+        // the staging of a short term table: many jobs with few batches each)
+        dp.tile_span = 1;
+        while (P.decode_files > 1 && P.terms_per_chunk <= dp.stage_terms && P.terms_per_chunk <= 16 &&
+               dp.tile_span < dp.tiles_per_seg && dp.tile_span < 8 &&
+               dp.nlist * P.nchunk * P.r * ((dp.tiles_per_seg + 2 * dp.tile_span - 1) / (2 * dp.tile_span)) >= (long long)P.sm_count * 16)
+            dp.tile_span *= 2;
+        dp.spans_per_seg = (dp.tiles_per_seg + dp.tile_span - 1) / dp.tile_span;
+        const long long blocks = dp.nlist * P.nchunk * P.r * dp.spans_per_seg;
         if (blocks > 0x7fffffffLL) return CCDC_ESIZE;
         const size_t smem = (size_t)dp.stage_terms * P.term_stride * sizeof(ccdc_ref);
-        // small r: the instantiation with r-1 as a compile-time constant
-        const int r1s = P.r <= 4 ? P.r - 1 : -1;
-        auto launch = [&](auto nt, auto r1, auto b1) {
+        // small r and 64- or 128-bit accesses: the instantiation with r-1 and the files loaded together
+        // as compile-time constants; everything else batch by batch
+        const int group = P.decode_files;
+        const bool fast = P.decode_files >= 1;
+        const int r1s = fast ? P.r - 1 : -1;
+        auto launch = [&](auto nt, auto r1, auto g) {
             constexpr int NT = decltype(nt)::value;
             constexpr int R1 = decltype(r1)::value;
-            constexpr bool B1 = decltype(b1)::value;
-            k_decode_reduce<VEC, F32, NT, R1, B1><<<(unsigned)blocks, NT, smem, st>>>(dp);
+            constexpr int G = decltype(g)::value;
+            launch_kernel(k_decode_reduce<VEC, F32, NT, R1, G>, blocks, NT, smem, st, dp);
         };
-        auto with_threads = [&](auto r1, auto b1) {
-            if (P.decode_threads == CCDC_DECODE_THREADS_SHORT) launch(std::integral_constant<int, CCDC_DECODE_THREADS_SHORT>(), r1, b1);
-            else launch(std::integral_constant<int, DTHREADS>(), r1, b1);
+        auto with_shape = [&](auto r1) {
+            constexpr int R1 = decltype(r1)::value;
+            constexpr bool GENERIC = R1 < 0;
+            const int nt = P.decode_threads;
+            if (!GENERIC && group == 4) launch(std::integral_constant<int, CCDC_DECODE_THREADS_FILES>(), r1, std::integral_constant<int, 4>());
+            else if (!GENERIC && group == 2) launch(std::integral_constant<int, CCDC_DECODE_THREADS_FILES>(), r1, std::integral_constant<int, 2>());
+            else if (nt == CCDC_DECODE_THREADS_SHORT) launch(std::integral_constant<int, CCDC_DECODE_THREADS_SHORT>(), r1, std::integral_constant<int, 1>());
+            else launch(std::integral_constant<int, DTHREADS>(), r1, std::integral_constant<int, 1>());
         };
-        // several files per batch: the batch-by-batch path measured faster (J-job workload, b = 7)
-        auto with_files = [&](auto r1) {
-            if (P.b == 1) with_threads(r1, std::true_type());
-            else with_threads(std::integral_constant<int, -1>(), std::false_type());
-        };
-        switch (r1s) {
-        case 0: with_files(std::integral_constant<int, 0>()); break;
-        case 1: with_files(std::integral_constant<int, 1>()); break;
-        case 2: with_files(std::integral_constant<int, 2>()); break;
-        case 3: with_files(std::integral_constant<int, 3>()); break;
-        default: with_threads(std::integral_constant<int, -1>(), std::false_type()); break;
+        if constexpr (VEC >= 2) {
+            switch (r1s) {
+            case 0: with_shape(std::integral_constant<int, 0>()); break;
+            case 1: with_shape(std::integral_constant<int, 1>()); break;
+            case 2: with_shape(std::integral_constant<int, 2>()); break;
+            case 3: with_shape(std::integral_constant<int, 3>()); break;
+            default: with_shape(std::integral_constant<int, -1>()); break;
+            }
+        } else {
+            with_shape(std::integral_constant<int, -1>());
         }
+        std::snprintf(g_last_decode, sizeof(g_last_decode), "k_decode_reduce<vec=%d,threads=%d,cancel=%d,files=%d,chunks=%d>",
+                      VEC, P.decode_threads, r1s, group, P.nchunk);
         int lrc = check_launch();
         if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
         const long long n = dp.nout * P.len, todo = dp.nlist * P.len;
-        k_sum_chunks<F32><<<(unsigned)((todo + DTHREADS - 1) / DTHREADS), DTHREADS, 0, st>>>(
-            dp.ws, dp.out, dp.out_rows, dp.nlist, P.len, n, P.nchunk);
+        launch_kernel(k_sum_chunks<F32>, (todo + DTHREADS - 1) / DTHREADS, DTHREADS, 0, st,
+               (const uint32_t *)dp.ws, dp.out, dp.out_rows, dp.nlist, P.len, n, P.nchunk);
         return check_launch();
     });
 }

@@ -87,35 +87,67 @@ int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
     return CCDC_OK;
 }
 
-// split of the batch loop of the fused decode over `nout` output rows: enough
-// thread blocks to fill the GPU (SMs x 8 resident blocks) while a block
-// still walks a fair number of batches.  P.sm_count is 148 (B200) until the
-// tables are uploaded, when the device's own count replaces it.
+// Launch shape of the fused decode over `nout` output rows: block size, files
+// of a batch whose loads are issued together, and the split of the batch loop
+// over blocks.  P.sm_count is 148 (B200) until the tables are uploaded, when
+// the device's own count replaces it.
+long long decode_tiles_per_seg(const ccdc_plan_s &P, int threads) {
+    const long long tile = (long long)threads * P.vec * CCDC_DECODE_VECTORS;
+    return (P.s + tile - 1) / tile;
+}
+
+void set_split(ccdc_plan_s &P, long long nchunk) {
+    nchunk = std::max(1LL, std::min(nchunk, P.nterm));
+    P.terms_per_chunk = (P.nterm + nchunk - 1) / nchunk;
+    P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
+}
+
 void choose_split(ccdc_plan_s &P, long long nout) {
-    auto split_for = [&](int threads, long long &per_chunk, int &nchunk) {
-        const long long tile = (long long)threads * P.vec * CCDC_DECODE_VECTORS;
-        const long long tiles_per_seg = (P.s + tile - 1) / tile;
-        const long long base = std::max(1LL, nout * P.r * tiles_per_seg);
+    // files of a batch loaded together: all of a small batch, fewer while a batch
+    // (coded word + r-1 operands) would keep more than 40 words per thread in flight
+    int group = P.b <= 1 ? 1 : P.b == 2 ? 2 : 4;
+    group = std::min(group, CCDC_DECODE_FILES_MAX);
+    while (group > 1 && (1 + (P.r - 1) * group) * P.vec > CCDC_DECODE_GROUP_WORDS) group /= 2;
+    if (P.r > 4 || P.vec < 2) group = 1;
+    // 0: the batch-by-batch kernel (any r, any number of files); 1: one-file batches
+    P.decode_files = (P.r > 4 || P.vec < 2 || (group == 1 && P.b > 1)) ? 0 : group;
+    // several files per batch: many registers per thread, so small blocks
+    P.decode_threads = group > 1 ? CCDC_DECODE_THREADS_FILES : CCDC_DECODE_THREADS;
+    // blocks resident per SM at the registers these kernels take
+    auto resident = [&](int threads) { return (long long)P.sm_count * (threads >= 1024 ? 1 : threads >= 512 ? 3 : 768 / threads); };
+    // enough thread blocks to fill the GPU (8 per SM) while a block still walks a fair number of batches
+    auto many_blocks = [&](int threads) {
+        const long long base = std::max(1LL, nout * P.r * decode_tiles_per_seg(P, threads));
         const long long want = ((long long)P.sm_count * 8 + base - 1) / base;
-        const long long cap = std::max(1LL, P.nterm / 8);
-        const long long nch = std::max(1LL, std::min(want, cap));
-        per_chunk = (P.nterm + nch - 1) / nch;
-        nchunk = (int)((P.nterm + per_chunk - 1) / per_chunk);
-        return base * nchunk;                       // thread blocks of the launch
+        return std::max(1LL, std::min(want, std::max(1LL, P.nterm / 8)));
     };
-    P.decode_threads = CCDC_DECODE_THREADS;
-    split_for(P.decode_threads, P.terms_per_chunk, P.nchunk);
-    // short segments: one large block per segment instead of two smaller ones, but only when the launch
-    // still has many waves of them (one such block is resident per SM); measured: K=16, r=4 gains 0.6 %,
-    // K=10, r=3 with 450 blocks would lose 17 %
-    if (P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
+    set_split(P, many_blocks(P.decode_threads));
+    const long long base = std::max(1LL, nout * P.r * decode_tiles_per_seg(P, P.decode_threads));
+    if (base * P.nchunk < 6 * resident(P.decode_threads)) {
+        // A launch of a few waves only: the rounding of the last wave decides.  Take the split with
+        // the fewest (waves x batches per block), a block costing two batches' time to start and end.
+        long long best = 0, best_cost = 0;
+        for (long long n = 1; n <= std::max(1LL, P.nterm / 4); ++n) {
+            const long long per = (P.nterm + n - 1) / n, real = (P.nterm + per - 1) / per;
+            if (real != n) continue;
+            const long long waves = (base * n + resident(P.decode_threads) - 1) / resident(P.decode_threads);
+            if (waves > 6) break;
+            const long long cost = waves * (per + 2);
+            if (best == 0 || cost < best_cost) { best = n; best_cost = cost; }
+        }
+        if (best) set_split(P, best);
+    }
+    // short segments of one-file batches: one large block per segment instead of two smaller ones, but only
+    // when the launch still has many waves of them (one such block is resident per SM); measured: K=16, r=4
+    // gains 0.6 %, K=10, r=3 with 450 blocks would lose 17 %
+    if (group <= 1 && P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
         P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS) {
-        long long per_chunk = 0;
-        int nchunk = 0;
-        if (split_for(CCDC_DECODE_THREADS_SHORT, per_chunk, nchunk) >= (long long)P.sm_count * 6) {
+        const long long n = many_blocks(CCDC_DECODE_THREADS_SHORT);
+        const long long per = (P.nterm + n - 1) / n, real = (P.nterm + per - 1) / per;
+        const long long blocks = nout * P.r * decode_tiles_per_seg(P, CCDC_DECODE_THREADS_SHORT) * real;
+        if (blocks >= (long long)P.sm_count * 6) {
             P.decode_threads = CCDC_DECODE_THREADS_SHORT;
-            P.terms_per_chunk = per_chunk;
-            P.nchunk = nchunk;
+            set_split(P, n);
         }
     }
 }
@@ -477,7 +509,7 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
             P.slot[(size_t)k * m + k % m] = 0;
             P.node_nfiles[k] = (k % m == m - 1) ? last : full;
         }
-        P.cmb.na = 1; P.cmb.n_max = P.len; P.cmb.uniform = false;
+        P.cmb.na = 1; P.cmb.n_max = P.len; P.cmb.uniform = false; P.cmb.nf_max = std::max(full, last);
         P.red_terms.resize((size_t)K * m);
         for (int k = 0; k < K; ++k) {
             int slot = 0;
@@ -507,7 +539,7 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
 void ccdc_internal_resplit(ccdc_plan_s *plan, int sm_count) {
     if (sm_count < 1 || sm_count == plan->sm_count) return;
     plan->sm_count = sm_count;
-    if (plan->compression_mode) return;
+    if (plan->compression_mode || plan->tuned) return;
     choose_split(*plan, plan->shard_world > 1 ? (long long)plan->out_rows.size() : plan->J * plan->K);
 }
 
@@ -561,6 +593,19 @@ void ccdc_plan_destroy(ccdc_plan_t *plan) {
     if (!plan) return;
     ccdc_internal_release_device(plan);
     delete plan;
+}
+
+int ccdc_plan_tune_decode(ccdc_plan_t *p, int threads, int chunks) {
+    if (!p) return CCDC_EINVAL;
+    if (p->compression_mode || p->device != -1) return CCDC_ESTATE;
+    if (chunks < 1 || chunks > p->nterm) return CCDC_EINVAL;
+    const bool files = p->decode_files > 1;
+    if (files ? threads != CCDC_DECODE_THREADS_FILES
+              : (threads != CCDC_DECODE_THREADS && threads != CCDC_DECODE_THREADS_SHORT)) return CCDC_EINVAL;
+    p->decode_threads = threads;
+    set_split(*p, chunks);
+    p->tuned = true;
+    return CCDC_OK;
 }
 
 int ccdc_plan_decode_threads(const ccdc_plan_t *p) { return p && !p->compression_mode ? p->decode_threads : 0; }

@@ -61,8 +61,10 @@ def assert_outputs(out_gpu, o, dtype):
     assert np.all(np.abs(got - s64) <= FP32_RTOL * a64 + 1e-30)
 
 
-def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0):
+def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0, tune=None):
     plan = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+    if tune:
+        plan.tune_decode(*tune)
     o = Oracle(K, r, N, Q, B, dtype, mode="paper" if jobs else "single")
     v = values_numpy(plan.J * N, Q, B, dtype, seed=seed, std=std)
     o.load_values(v)
@@ -137,6 +139,10 @@ SHAPES = [
     (3, 1, 30, 3, 2100),                    # b = 10, r = 1: one operand, eight files' loads in flight
     (5, 3, 50, 5, 777),                     # b = 5, three operands
     (5, 4, 15, 5, 1300),                    # b = 3, four operands
+    (6, 2, 15, 6, 65544),                   # b = 1, segments of 32 772 words: the 512-thread form of the fused encode
+    (4, 2, 6, 8, 6 * 1366 + 2),             # Q/K = 2, b = 1, ragged
+    (6, 2, 105, 6, 3000),                   # b = 7: two groups of files per operand (4 + 3)
+    (5, 1, 45, 5, 2200),                    # b = 9, r = 1: three groups, no cancel operand
 ]
 
 
@@ -175,6 +181,30 @@ def test_cfg3_short_values(ccdc):
 def test_cfg4_short_values(ccdc):
     w = CONFIGS["cfg4"].scaled(6000)
     run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype, std=w.std)
+
+
+def test_cfg3_structure_exhaustive_1024_thread_decode(ccdc):
+    """K=16, r=4, N=1820, Q=16 with values of 8208 elements: segments of 2052 words select the
+    1024-thread block of the fused decode, the launch shape of the full-size workload; every coded
+    word, packet and output against the oracle."""
+    w = CONFIGS["cfg3"].scaled(8208)
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
+    assert plan.decode_threads == 1024 and plan.decode_chunks > 1
+    assert "threads=1024" in ccdc.last_decode_kernel() and "cancel=3" in ccdc.last_decode_kernel()
+    full = ccdc.Plan(w.K, w.r, w.N, w.Q, CONFIGS["cfg3"].B, w.dtype)
+    assert (full.decode_threads, full.decode_chunks) == (plan.decode_threads, plan.decode_chunks)
+
+
+def test_cfg4_structure_exhaustive_wide_encode(ccdc):
+    """K=20, r=2, N=190, Q=20 with values of 65 544 elements: one-file rows of 32 772 words select the
+    512-thread form of the fused encode with several tiles per block and a ragged last tile, the
+    launch shape of the full-size workload; every coded word, packet and output against the oracle."""
+    w = CONFIGS["cfg4"].scaled(65544)
+    full = ccdc.Plan(w.K, w.r, w.N, w.Q, CONFIGS["cfg4"].B, w.dtype)
+    assert (full.decode_threads, full.decode_chunks) == (512, 1)
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype, std=w.std, tune=(512, 1))   # the full size's decode shape
+    assert "operands=2,files=1,vectors=2,threads=512" in ccdc.last_gather_kernel()
+    assert "threads=512,cancel=1,files=1,chunks=1" in ccdc.last_decode_kernel()
 
 
 def test_cfg5_shuffle_shape(ccdc):
@@ -365,8 +395,15 @@ def sampled_full_size_check(ccdc, w, offsets_per_segment=48, seed=5):
     plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
     s = plan.segment_elems
     rng = np.random.default_rng(seed)
-    tile = 2048
-    fixed = [0, 1, 3, s - 1, s - 4, min(tile - 1, s - 1), min(tile, s - 1), s // 2]
+    # first and last word of a tile and of a block's span for every tile the two launches use at these
+    # shapes (the fused encode: 256 or 512 threads x 4 words x 2 vectors, 32 tiles per block; the fused
+    # decode: 512 or 1024 threads x 4 words), and of the ragged last tile and span
+    fixed = [0, 1, 3, s - 1, s - 4, s // 2]
+    for tile in (2048, 4096):
+        span = 32 * tile
+        for edge in (tile, 2 * tile, span, (s - 1) // tile * tile, (s - 1) // span * span):
+            fixed += [edge - 1, edge]
+    fixed = [x for x in fixed if 0 <= x < s]
     offs = np.unique(np.concatenate([np.array(fixed), rng.integers(0, s, offsets_per_segment)]))
     m = len(offs)
     index = np.concatenate([i * s + offs for i in range(w.r)])
@@ -399,11 +436,108 @@ def sampled_full_size_check(ccdc, w, offsets_per_segment=48, seed=5):
 
 
 def test_cfg3_full_size_sampled(ccdc):
-    sampled_full_size_check(ccdc, CONFIGS["cfg3"])
+    plan = sampled_full_size_check(ccdc, CONFIGS["cfg3"])
+    assert "threads=1024" in ccdc.last_decode_kernel()
+    assert plan.coded_bits == 2_862_612_480
 
 
 def test_cfg4_full_size_sampled(ccdc):
     free, _ = torch.cuda.mem_get_info()
     if free < 60 * 2**30:
         pytest.fail("cfg4 needs about 50 GB of device memory")
-    sampled_full_size_check(ccdc, CONFIGS["cfg4"], offsets_per_segment=24)
+    plan = sampled_full_size_check(ccdc, CONFIGS["cfg4"], offsets_per_segment=24)
+    assert "threads=512" in ccdc.last_gather_kernel() and "threads=512" in ccdc.last_decode_kernel()
+    assert plan.coded_bits == 70_041_600_000
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", [(4, 2, 12, 4, 300), (10, 3, 480, 10, 96), (6, 3, 20, 12, 2049)])
+def test_shuffle_from_host_buffers(ccdc, K, r, N, Q, B, dtype):
+    """ccdc_shuffle_host: Map results in pinned host memory, outputs back in host memory, copies and
+    the two launches on one stream; outputs and the coded rows left on the device against the oracle."""
+    plan = ccdc.Plan(K, r, N, Q, B, dtype)
+    o = Oracle(K, r, N, Q, B, dtype)
+    v = values_numpy(N, Q, B, dtype, seed=77)
+    o.load_values(v)
+    o.shuffle()
+    row = Q * B
+    host_part = []
+    for k in range(K):
+        files = plan.node_files(k)
+        h = torch.empty(len(files) * row, dtype=plan.torch_dtype).pin_memory()
+        h.view(-1, row).copy_(torch.from_numpy(v.reshape(N, row)[files]))
+        host_part.append(h)
+    host_out = torch.full((Q * B,), 7, dtype=plan.torch_dtype).pin_memory()
+    part = plan.alloc_partitions()
+    coded_w, coded = guarded(plan.coded_bytes // 4, plan.torch_dtype)
+    out_w, out = guarded(Q * B, plan.torch_dtype)
+    ws = plan.alloc(plan.workspace_bytes)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(2):          # the second call finds the first one's data everywhere
+            plan.shuffle_host(host_part, host_out, part, coded, out, ws if ws.numel() else None, stream=stream)
+    stream.synchronize()
+    s, sp = plan.segment_elems, plan.coded_row_elems
+    assert np.array_equal(bits(coded).reshape(-1, sp)[:, :s], o.coded().reshape(-1, s))
+    assert canaries_intact(coded_w, plan.coded_bytes // 4) and canaries_intact(out_w, Q * B)
+    assert_outputs(host_out, o, dtype)
+    assert torch.equal(host_out, out.cpu())
+    for k in range(K):
+        assert torch.equal(part[k].cpu(), host_part[k])
+
+
+@pytest.mark.parametrize("K,r,N,Q,B,jobs", [(5, 2, 10, 5, 1000, False), (10, 3, 480, 10, 64, False),
+                                            (4, 2, 12, 8, 37, False), (5, 2, 9, 5, 50, True)])
+def test_words_written_by_the_encode_are_the_multicast_bits(ccdc, K, r, N, Q, B, jobs):
+    """Definition 1 counted on the device: the coded buffer starts full of a word no coded word can
+    equal (Map values below 2**20, so every sum and XOR stays below 2**31; the mark has bit 31 set);
+    after the fused encode the words that changed, times 32, are the plan's multicast bit count."""
+    plan = ccdc.Plan(K, r, N, Q, B, "int32", jobs=jobs)
+    v = (values_numpy(plan.J * N, Q, B, "int32", seed=9).view(np.uint32) >> 12).view(np.int32)
+    part = plan.alloc_partitions()
+    plan.fill_partitions(part, torch.from_numpy(v).cuda())
+    mark = -0x7A5A5A5B      # bit 31 set
+    coded = torch.full((plan.coded_bytes // 4,), mark, dtype=torch.int32, device="cuda")
+    plan.encode_fused(part, coded)
+    torch.cuda.synchronize()
+    written = int((coded != mark).sum().item())
+    assert written * 32 == plan.coded_bits
+    o = Oracle(K, r, N, Q, B, "int32", mode="paper" if jobs else "single")
+    o.load_values(v)
+    o.shuffle()
+    assert written * 32 == o.coded_bits
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+def test_decode_shape_overrides_keep_parity(ccdc, dtype):
+    """ccdc_plan_tune_decode: every allowed launch shape of the fused decode gives the oracle's outputs."""
+    for (K, r, N, Q, B), shapes in (((10, 3, 480, 10, 96), [(128, c) for c in (1, 2, 7, 15, 120)]),
+                                    ((6, 2, 15, 6, 9000), [(512, 1), (512, 3), (1024, 2), (1024, 15)])):
+        o = Oracle(K, r, N, Q, B, dtype)
+        v = values_numpy(N, Q, B, dtype, seed=K)
+        o.load_values(v)
+        o.shuffle()
+        for threads, chunks in shapes:
+            plan = ccdc.Plan(K, r, N, Q, B, dtype)
+            plan.tune_decode(threads, chunks)
+            assert (plan.decode_threads, plan.decode_chunks) == (threads, chunks)
+            part = plan.alloc_partitions()
+            plan.fill_partitions(part, torch.from_numpy(v).cuda())
+            coded = plan.alloc(plan.coded_bytes)
+            out_w, out = guarded(Q * B, plan.torch_dtype)
+            ws_w, ws = guarded(plan.workspace_bytes // 4, plan.torch_dtype)
+            assert (plan.workspace_bytes > 0) == (chunks > 1)
+            for _ in range(2):      # the counters of the split loop must be back at zero for the second call
+                plan.shuffle(part, coded, out, ws if plan.workspace_bytes else None)
+            torch.cuda.synchronize()
+            assert canaries_intact(out_w, Q * B) and canaries_intact(ws_w, plan.workspace_bytes // 4)
+            assert_outputs(out, o, dtype)
+            assert f"threads={threads}" in ccdc.last_decode_kernel() and f"chunks={chunks}" in ccdc.last_decode_kernel()
+            with pytest.raises(ccdc.CcdcError) as e:
+                plan.tune_decode(threads, chunks)           # the tables are on the device now
+            assert e.value.status == ccdc.ESTATE
+    bad = ccdc.Plan(10, 3, 480, 10, 96, dtype)
+    for threads, chunks in ((512, 4), (128, 0), (128, 121)):
+        with pytest.raises(ccdc.CcdcError) as e:
+            bad.tune_decode(threads, chunks)
+        assert e.value.status == ccdc.EINVAL
