@@ -95,6 +95,14 @@ typedef enum {
  * Host only: no CUDA call is made.  Destroy with ccdc_plan_destroy. */
 int  ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
 int  ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out);
+/* ccdc_plan_jobs_gamma: J = gamma * C(K,r+1) jobs (Section IV: "repeats the same
+ * operations gamma times"), all shuffled by the same two launches.  Job j lives
+ * on subset j mod C(K,r+1); jobs g*C(K,r+1) .. (g+1)*C(K,r+1)-1 form group g, an
+ * independent instance of ccdc_plan_jobs whose batches, rounds, files (global id
+ * j*N + n), functions and outputs follow those of group g-1 in every layout.
+ * gamma >= 1 (CCDC_EINVAL otherwise); gamma = 1 is ccdc_plan_jobs. */
+int  ccdc_plan_jobs_gamma(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, int gamma,
+                          ccdc_plan_t **out);
 /* ccdc_plan_compression: the compression-only scheme of the paper's appendix
  * ("Communication Load of the compression scheme"), kept as a measured
  * comparator.  One job, mu = r/K: the files are cut into m = ceil(K/r) batches,
@@ -341,6 +349,60 @@ int ccdc_job_host(ccdc_plan_t *plan, const void *const *host_x, const void *cons
                   long long rows, void *host_out, void *const *dev_x, void *const *dev_y, void *dev_w,
                   void *const *dev_part, void *dev_coded, void *dev_out, void *map_workspace, void *dev_workspace,
                   void *stream);
+
+/* --------------------------------------------------------- several GPUs
+ * One process per GPU.  The shuffle shards two ways; neither makes a kernel of
+ * one GPU wait for another GPU.
+ *
+ * (1) Value-dimension shards, no exchange.  Every step of Section IV-B (sums,
+ * XORs, cancellations) acts on words at equal positions of equal-size
+ * segments, so GPU `rank` of `world` can own the sub-range [rank*w, (rank+1)*w),
+ * w = s/world, of EVERY segment of every packet and run the complete scheme on
+ * it: an exact instance of the scheme with values of B_local = r*w/(Q/K)
+ * elements.  Requires r | (Q/K)*B, world | s and (Q/K) | r*w (CCDC_EINVAL
+ * otherwise).  Each rank makes an ordinary plan ccdc_plan(K, r, N, Q, B_local)
+ * (or ccdc_plan_jobs) and shuffles alone; the multicast bits of the ranks add
+ * up to those of the unsharded job.
+ *   ccdc_value_shard           B_local for this rank (host only).
+ *   ccdc_value_shard_position  position in the full packet ((Q/K)*B words) of
+ *                              word local_pos of the rank's packet (r*w words);
+ *                              -1 if out of range (host only).
+ *   ccdc_value_shard_copy      device copy between the full layout
+ *                              [rows][Q][B] and the rank's [rows][Q][B_local]
+ *                              (rows = files for Map results, jobs for
+ *                              outputs): to_local != 0 gathers the rank's words
+ *                              out of `src` (full) into `dst` (local); to_local
+ *                              = 0 scatters `src` (local) to the rank's
+ *                              positions of `dst` (full), leaving the rest of
+ *                              dst untouched.  One launch on `stream`.  A Map
+ *                              that runs per rank would write its slice
+ *                              directly; the copy serves tests and callers
+ *                              that hold full-length values. */
+int ccdc_value_shard(int K, int r, int Q, long long B, int rank, int world, long long *B_local);
+long long ccdc_value_shard_position(int K, int r, int Q, long long B, int rank, int world, long long local_pos);
+int ccdc_value_shard_copy(int K, int r, int Q, long long B, int rank, int world, int to_local, const void *src,
+                          void *dst, long long rows, void *stream);
+
+/* (2) Node shards with peer stores (ccdc_plan_sharded + ccdc_encode_fused_peers,
+ * above): the multicast of Section IV-B as plain stores into every rank's coded
+ * buffer.  For that each rank's buffer must be addressable from the other
+ * processes: ccdc_peer_buffer_create allocates `bytes` of device memory on the
+ * current device and fills handle_out (CCDC_PEER_HANDLE_BYTES bytes, to be sent
+ * to the other ranks by any host channel); ccdc_peer_buffer_open maps another
+ * process's buffer into this one (peer access is enabled as needed) and
+ * ccdc_peer_buffer_close unmaps it; ccdc_peer_buffer_destroy frees one's own
+ * buffer after the others closed it.  ccdc_peer_buffer_copy is an asynchronous
+ * copy between any two of device, peer and host memory (direction inferred).
+ * These calls allocate and synchronise: set-up and tear-down, not the data
+ * path.  The data path stays plain peer stores by the encode kernel; the ranks
+ * synchronise on the host (or with a collective on the stream) between the
+ * encode and the decode launch. */
+#define CCDC_PEER_HANDLE_BYTES 64
+int ccdc_peer_buffer_create(size_t bytes, void **dev_ptr, void *handle_out);
+int ccdc_peer_buffer_open(const void *handle, void **dev_ptr);
+int ccdc_peer_buffer_close(void *dev_ptr);
+int ccdc_peer_buffer_destroy(void *dev_ptr);
+int ccdc_peer_buffer_copy(void *dst, const void *src, size_t bytes, void *stream);
 
 /* Allocation-free variant of ccdc_decode_reduce (the paper has no counterpart:
  * this is a property of the library, not a step of the scheme).

@@ -10,12 +10,12 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libccdc.so"
-SOURCES = ["ccdc_plan.cpp", "ccdc_kernels.cu", "ccdc_map.cu", "ccdc_map_cluster.cu"]
+SOURCES = ["ccdc_plan.cpp", "ccdc_kernels.cu", "ccdc_map.cu", "ccdc_map_cluster.cu", "ccdc_multi.cu"]
 
 
 def nvcc_command(out: Path, verbose: bool = False, defines: tuple[str, ...] = ()) -> list[str]:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
+    cmd = [nvcc, "-O3", "-std=c++17", "--threads", "0", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
            "-Xcompiler", "-fPIC,-Wall", "-shared", "-cudart", "static",
            "-I", str(ROOT / "include"), "-I", str(CSRC), "-o", str(out)]
     if verbose:

@@ -27,6 +27,7 @@ _PP = ctypes.POINTER(ctypes.c_void_p)
 SIGNATURES = {
     "ccdc_plan": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_jobs": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
+    "ccdc_plan_jobs_gamma": (_I, [_I, _I, _LL, _I, _LL, _I, _I, _PP]),
     "ccdc_plan_compression": (_I, [_I, _I, _LL, _I, _LL, _I, _PP]),
     "ccdc_plan_sharded": (_I, [_I, _I, _LL, _I, _LL, _I, _I, _I, _I, _PP]),
     "ccdc_plan_coded_row_position": (_LL, [_P, _LL, _I]),
@@ -74,6 +75,14 @@ SIGNATURES = {
     "ccdc_compression_shuffle": (_I, [_P, _PP, _PP, _P, _P]),
     "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
     "ccdc_job_host": (_I, [_P, _PP, _PP, _P, _LL, _P, _PP, _PP, _P, _PP, _P, _P, _P, _P, _P]),
+    "ccdc_value_shard": (_I, [_I, _I, _I, _LL, _I, _I, ctypes.POINTER(ctypes.c_longlong)]),
+    "ccdc_value_shard_position": (_LL, [_I, _I, _I, _LL, _I, _I, _LL]),
+    "ccdc_value_shard_copy": (_I, [_I, _I, _I, _LL, _I, _I, _I, _P, _P, _LL, _P]),
+    "ccdc_peer_buffer_create": (_I, [_SZ, _PP, _P]),
+    "ccdc_peer_buffer_open": (_I, [_P, _PP]),
+    "ccdc_peer_buffer_close": (_I, [_P]),
+    "ccdc_peer_buffer_destroy": (_I, [_P]),
+    "ccdc_peer_buffer_copy": (_I, [_P, _P, _SZ, _P]),
     "ccdc_strerror": (ctypes.c_char_p, [_I]),
     "ccdc_last_cuda_error": (_I, []),
     "ccdc_num_kernel_launches": (_I, []),
@@ -117,6 +126,67 @@ def _ptr_array(tensors):
     return arr
 
 
+PEER_HANDLE_BYTES = 64
+
+
+class PeerBuffer:
+    """Device memory that another process can open (``ccdc_peer_buffer_*``).  Quacks like a tensor
+    for the step calls (``data_ptr`` / ``numel``).  ``PeerBuffer.create(nbytes)`` allocates on the
+    current device and exposes ``handle`` (64 bytes to send to the other ranks);
+    ``PeerBuffer.open(handle, nbytes)`` maps another process's buffer."""
+
+    def __init__(self, ptr, nbytes, handle, owner):
+        self.ptr, self.nbytes, self.handle, self.owner = ptr, nbytes, handle, owner
+
+    @classmethod
+    def create(cls, nbytes):
+        ptr = ctypes.c_void_p()
+        handle = (ctypes.c_ubyte * PEER_HANDLE_BYTES)()
+        _check(lib().ccdc_peer_buffer_create(nbytes, ctypes.byref(ptr), handle), "ccdc_peer_buffer_create")
+        return cls(ptr.value, nbytes, bytes(handle), True)
+
+    @classmethod
+    def open(cls, handle, nbytes):
+        ptr = ctypes.c_void_p()
+        buf = (ctypes.c_ubyte * PEER_HANDLE_BYTES).from_buffer_copy(handle)
+        _check(lib().ccdc_peer_buffer_open(buf, ctypes.byref(ptr)), "ccdc_peer_buffer_open")
+        return cls(ptr.value, nbytes, bytes(handle), False)
+
+    def data_ptr(self):
+        return self.ptr
+
+    def numel(self):
+        return self.nbytes // 4
+
+    def copy_to(self, tensor, stream=None):
+        """copies the buffer into a tensor (device or pinned host) of the same size."""
+        _check(lib().ccdc_peer_buffer_copy(tensor.data_ptr(), self.ptr, self.nbytes, _stream_handle(stream)),
+               "ccdc_peer_buffer_copy")
+
+    def release(self):
+        if self.ptr:
+            fn = lib().ccdc_peer_buffer_destroy if self.owner else lib().ccdc_peer_buffer_close
+            _check(fn(self.ptr), "ccdc_peer_buffer_release")
+            self.ptr = None
+
+
+def value_shard(K, r, Q, B, rank, world) -> int:
+    """value length of rank's shard when every segment is cut into `world` sub-ranges."""
+    out = ctypes.c_longlong()
+    _check(lib().ccdc_value_shard(K, r, Q, B, rank, world, ctypes.byref(out)), "ccdc_value_shard")
+    return out.value
+
+
+def value_shard_position(K, r, Q, B, rank, world, local_pos) -> int:
+    return lib().ccdc_value_shard_position(K, r, Q, B, rank, world, local_pos)
+
+
+def value_shard_copy(K, r, Q, B, rank, world, to_local, src, dst, rows, stream=None):
+    """device copy between the full layout [rows][Q][B] and the rank's [rows][Q][B_local]."""
+    _check(lib().ccdc_value_shard_copy(K, r, Q, B, rank, world, int(to_local), src.data_ptr(), dst.data_ptr(), rows,
+                                       _stream_handle(stream)), "ccdc_value_shard_copy")
+
+
 def _stream_handle(stream):
     import torch
 
@@ -127,7 +197,7 @@ def _stream_handle(stream):
 class Plan:
     """``ccdc_plan`` / ``ccdc_plan_jobs`` plus the step calls on torch tensors."""
 
-    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False, compression: bool = False, shard=None):
+    def __init__(self, K, r, N, Q, B, dtype, jobs: bool = False, compression: bool = False, shard=None, gamma: int = 1):
         self.K, self.r, self.N, self.Q, self.B = K, r, N, Q, B
         self.dtype = {"int32": I32, "float32": F32, I32: I32, F32: F32}[dtype]
         self.jobs = jobs
@@ -138,6 +208,10 @@ class Plan:
         if shard is not None:           # (rank, world): this GPU's share of the logical nodes
             _check(lib().ccdc_plan_sharded(K, r, N, Q, B, self.dtype, int(jobs), shard[0], shard[1], ctypes.byref(h)),
                    "ccdc_plan_sharded")
+        elif gamma != 1:
+            if not jobs:
+                raise ValueError("gamma > 1 belongs to the J-job scheme (jobs=True)")
+            _check(lib().ccdc_plan_jobs_gamma(K, r, N, Q, B, self.dtype, gamma, ctypes.byref(h)), "ccdc_plan_jobs_gamma")
         else:
             _check(fn(K, r, N, Q, B, self.dtype, ctypes.byref(h)), "ccdc_plan")
         self._h = h

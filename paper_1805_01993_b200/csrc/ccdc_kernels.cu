@@ -617,7 +617,14 @@ k_sum_chunks(const uint32_t *__restrict__ ws, uint32_t *__restrict__ out, const 
     pdl_trigger();
     pdl_wait();
     uint32_t acc = ws[e];
-    for (int c = 1; c < nchunk; ++c) acc = add_word<F32>(acc, ws[(long long)c * n + e]);
+    for (int c = 1; c < nchunk; c += 8) {           // eight chunks' loads in flight, added in chunk order
+        uint32_t w[8];
+#pragma unroll
+        for (int x = 0; x < 8; ++x) w[x] = c + x < nchunk ? ws[(long long)(c + x) * n + e] : 0u;
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+            if (c + x < nchunk) acc = add_word<F32>(acc, w[x]);
+    }
     out[e] = acc;
 }
 

@@ -383,7 +383,8 @@ int finish(ccdc_plan_s &P) {
     return CCDC_OK;
 }
 
-int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, bool jobs, ccdc_plan_t **out) {
+int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, bool jobs, ccdc_plan_t **out,
+              int gamma = 1) {
     if (!out) return CCDC_EINVAL;
     *out = nullptr;
     int rc = check_parameters(K, r, N, Q, B, (int)dtype);
@@ -392,6 +393,8 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
     if (n_rsub <= 0 || n_r1sub <= 0 || n_r1sub > (1LL << 24)) return CCDC_ESIZE;
     if (!jobs && N % n_rsub != 0) return CCDC_EINVAL;       // batches of equal size
     if (jobs && N % (r + 1) != 0) return CCDC_EINVAL;
+    if (gamma < 1 || (!jobs && gamma != 1)) return CCDC_EINVAL;
+    if ((long long)gamma * n_r1sub > (1LL << 24)) return CCDC_ESIZE;
     try {
         ccdc_plan_s *pp = new ccdc_plan_s();
         ccdc_plan_s &P = *pp;
@@ -421,7 +424,9 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
                 }
             }
         } else {
-            P.J = n_r1sub; P.b = N / (r + 1); P.nbatch = P.J * (r + 1); P.nround = P.J * (K - r);
+            // gamma groups of C(K, r+1) jobs: job j lives on subset j mod C(K, r+1); the groups are
+            // independent repetitions of the same operations (Section IV: J = gamma * C(K, mu K + 1))
+            P.J = (long long)gamma * n_r1sub; P.b = N / (r + 1); P.nbatch = P.J * (r + 1); P.nround = P.J * (K - r);
             P.nterm = r + 1;
             P.job_batch0.resize(P.J);
             P.batch_nodes.resize((size_t)P.nbatch * r);
@@ -429,7 +434,7 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
             // the a-th size-r subset of an (r+1)-set in lexicographic order
             // omits its (r-a)-th member
             for (long long j = 0; j < P.J; ++j) {
-                subset_unrank(j, r + 1, K, c);
+                subset_unrank(j % n_r1sub, r + 1, K, c);
                 P.job_batch0[j] = j * (r + 1);
                 for (int a = 0; a <= r; ++a) {
                     const long long p = j * (r + 1) + a;
@@ -442,7 +447,8 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
             P.round_batch.resize((size_t)P.nround * (r + 1));
             long long g = 0;
             for (long long j = 0; j < P.J; ++j) {
-                subset_unrank(j, r + 1, K, c);
+                subset_unrank(j % n_r1sub, r + 1, K, c);
+                const long long group0 = j / n_r1sub * n_r1sub;     // first job of j's group
                 // stage 1: member a receives job j's batch that omits it
                 std::memcpy(&P.round_group[(size_t)g * (r + 1)], c, sizeof(int) * (r + 1));
                 for (int a = 0; a <= r; ++a) P.round_batch[(size_t)g * (r + 1) + a] = j * (r + 1) + (r - a);
@@ -461,7 +467,7 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
                             rest[y++] = c[x];
                         }
                         if (!placed) { m = y; rest[y++] = i; }
-                        const long long jt = subset_rank(rest, r + 1, K);
+                        const long long jt = group0 + subset_rank(rest, r + 1, K);
                         P.round_batch[(size_t)g * (r + 1) + a] = jt * (r + 1) + (r - m);
                     }
                     ++g;
@@ -587,6 +593,11 @@ int ccdc_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
 
 int ccdc_plan_jobs(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, ccdc_plan_t **out) {
     return make_plan(K, r, N, Q, B, dtype, true, out);
+}
+
+int ccdc_plan_jobs_gamma(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype, int gamma,
+                         ccdc_plan_t **out) {
+    return make_plan(K, r, N, Q, B, dtype, true, out, gamma);
 }
 
 void ccdc_plan_destroy(ccdc_plan_t *plan) {

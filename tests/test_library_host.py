@@ -165,3 +165,75 @@ def test_node_sharded_plans_agree_on_the_gathered_layout(K, r, N, world, jobs):
         assert pl.coded_bits == full.coded_bits        # what crosses between the GPUs is the multicast load
     with pytest.raises(ccdc.CcdcError):
         ccdc.Plan(6, 2, 15, 6, 8, "int32", shard=(0, 4))     # world must divide K
+
+
+@pytest.mark.parametrize("K,r,N,gamma", [(4, 2, 6, 2), (5, 2, 9, 3), (5, 3, 8, 2)])
+def test_gamma_groups_repeat_the_jobs_plan(K, r, N, gamma):
+    """J = gamma * C(K, r+1) jobs: group g is the oracle's J-job plan with every batch, round,
+    job and file id moved on by g groups; the multicast bits are gamma times one group's, so the
+    load per J*Q*T is still Theorem 1."""
+    from fractions import Fraction
+
+    Q, B = K, 6
+    p = ccdc.Plan(K, r, N, Q, B, "int32", jobs=True, gamma=gamma)
+    o = Oracle(K, r, N, Q, B, "int32", mode="paper")
+    assert (p.J, p.num_batches, p.num_groups, p.files_per_batch) == (gamma * o.J, gamma * o.nbatch, gamma * o.nround, o.b)
+    for g in range(gamma):
+        for b in range(o.nbatch):
+            nodes, f0, job = p.batch(g * o.nbatch + b)
+            assert nodes == o.batch_nodes(b) and job == g * o.J + o.batch_job(b)
+            assert f0 == g * o.J * N + o.batch_files(b)[0]
+        for rd in range(o.nround):
+            assert p.group(g * o.nround + rd) == o.round_group(rd)
+            assert p.group_batches(g * o.nround + rd) == [g * o.nbatch + x for x in o.round_batches(rd)]
+    assert p.coded_bits == gamma * o.nround * (r + 1) * 32 * o.s
+    assert Fraction(p.coded_bits, p.J * Q * 32 * B) == Fraction((K - r) * (r + 1), K * r) * Fraction(r * o.s, o.len)
+    assert p.out_bytes == gamma * o.J * Q * B * 4
+    for k in range(K):
+        assert p.partition_bytes(k) == gamma * o.node_num_files(k) * Q * B * 4
+    with pytest.raises(ccdc.CcdcError):
+        ccdc.Plan(K, r, N, Q, B, "int32", jobs=True, gamma=0)
+    with pytest.raises(ValueError):
+        ccdc.Plan(K, r, comb(K, r), Q, B, "int32", gamma=2)
+
+
+@pytest.mark.parametrize("K,r,Q,B,world", [(4, 2, 4, 16, 2), (6, 3, 12, 30, 5), (10, 2, 10, 64, 4), (5, 1, 5, 12, 3)])
+def test_value_shards_partition_every_segment(K, r, Q, B, world):
+    """Rank g owns sub-range g of every segment: the ranks' position maps are disjoint, cover the
+    packet, keep a word inside its segment and at the same offset in every segment."""
+    length = (Q // K) * B
+    s = length // r
+    w = s // world
+    seen = []
+    for rank in range(world):
+        b_local = ccdc.value_shard(K, r, Q, B, rank, world)
+        assert b_local * (Q // K) == r * w
+        pos = [ccdc.value_shard_position(K, r, Q, B, rank, world, x) for x in range(r * w)]
+        assert ccdc.value_shard_position(K, r, Q, B, rank, world, r * w) == -1
+        for x, full in enumerate(pos):
+            i, off = divmod(x, w)
+            assert full // s == i and full % s == rank * w + off
+        seen += pos
+    assert sorted(seen) == list(range(length))
+    for bad in ((K, r, Q, B + 1, 0, world), (K, r, Q, B, world, world), (K, r, Q, B, 0, 7 * s + 1)):
+        with pytest.raises(ccdc.CcdcError) as e:
+            ccdc.value_shard(*bad)
+        assert e.value.status == ccdc.EINVAL
+
+
+def test_decode_shape_queries_and_override():
+    """The planner's launch shape of the fused decode, for the five workloads, and its override."""
+    shapes = {(4, 2, 12, 4, 256): (128, 1), (16, 4, 1820, 16, 16384): (1024, 19), (20, 2, 190, 20, 1_280_000): (512, 1)}
+    for shape, want in shapes.items():
+        p = ccdc.Plan(*shape, "float32")
+        assert (p.decode_threads, p.decode_chunks) == want, shape
+        assert (p.workspace_bytes > 0) == (p.decode_chunks > 1)
+    p = ccdc.Plan(10, 3, 480, 10, 4096, "float32")
+    assert p.decode_threads == 128 and 1 < p.decode_chunks <= 15
+    p.tune_decode(128, 6)
+    assert p.decode_chunks == 6 and p.workspace_bytes == 6 * 10 * 4096 * 4
+    for threads, chunks in ((256, 6), (128, 0), (128, 121)):
+        with pytest.raises(ccdc.CcdcError) as e:
+            p.tune_decode(threads, chunks)
+        assert e.value.status == ccdc.EINVAL
+    assert ccdc.last_gather_kernel() == "" or "k_gather" in ccdc.last_gather_kernel()
