@@ -294,7 +294,19 @@ def run_ours(args, w):
     sharded = bool(args.shard_nodes) and world > 1
     if sharded and (w.map_rows or w.K % world):
         raise RuntimeError("--shard-nodes needs a shuffle-only workload and a GPU count that divides K")
+    # --shard-values: ONE job over all GPUs, every GPU owning one sub-range of every segment: each rank
+    # runs the whole scheme on values of B/N elements, nothing is exchanged (strong scaling).
+    value_sharded = bool(args.shard_values) and world > 1
+    full_B = w.B
+    if value_sharded:
+        if sharded or w.map_rows:
+            raise RuntimeError("--shard-values is for the shuffle-only workloads and excludes --shard-nodes")
+        w = w.scaled(ccdc.value_shard(w.K, w.r, w.Q, w.B, rank, world))
     plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=w.jobs, shard=(rank, world) if sharded else None)
+    if args.family is not None:
+        plan.tune_family(args.family)
+    if args.decode_chunks:
+        plan.tune_decode(plan.decode_threads, args.decode_chunks)
     plan.upload()
     part = plan.alloc_partitions(dev)
     coded = plan.alloc(plan.coded_bytes, dev)
@@ -327,7 +339,34 @@ def run_ours(args, w):
         # every rank is an independent job of the same shape: its own seed
         plan.fill_partitions_streaming(part, values_torch(plan.J * w.N, w.Q, w.B, w.dtype, dev, seed=rank_seed(rank),
                                                           std=w.std))
+    wire = None
     if sharded:
+        # Definition 1 counts a multicast once; between GPUs a coded row has to reach every OTHER GPU
+        # that hosts one of its receivers.  The all-gather (and the peer stores) deliver every row to
+        # all world-1 other GPUs.
+        per = w.K // world
+        needed = 0
+        for g in range(plan.num_groups):
+            members = plan.group(g)
+            for a, sender in enumerate(members):
+                needed += len({k // per for k in members if k != sender} - {sender // per})
+        row_bytes = plan.segment_elems * 4
+        wire = {"multicast_bytes": plan.coded_bits // 8,
+                "wire_bytes_per_step": plan.num_groups * (w.r + 1) * row_bytes * (world - 1),
+                "needed_wire_bytes_per_step": needed * row_bytes,
+                "exchange": "peer stores by the encode kernel" if args.peer_stores else "NCCL all-gather of the send buffers"}
+    if sharded and args.peer_stores:
+        # every rank's coded buffer opened in every process; the encode kernel stores each row it
+        # produces into all of them, an all-reduce of one word orders the ranks before the decode
+        mine = ccdc.PeerBuffer.create(plan.coded_bytes)
+        handles = [None] * world
+        dist.all_gather_object(handles, mine.handle)
+        peers = [mine if d == rank else ccdc.PeerBuffer.open(handles[d], plan.coded_bytes) for d in range(world)]
+        coded = mine
+        token = torch.zeros(1, device=dev)
+        stages.append(("k_gather(encode)", lambda: plan.encode_fused_peers(part, peers)))
+        stages.append(("all_gather(coded rows)", lambda: dist.all_reduce(token)))
+    elif sharded:
         send = plan.alloc(plan.coded_send_bytes, dev)
         stages.append(("k_gather(encode)", lambda: plan.encode_fused(part, send)))
         stages.append(("all_gather(coded rows)", lambda: dist.all_gather_into_tensor(coded, send)))
@@ -423,6 +462,7 @@ def run_ours(args, w):
             raise
         except Exception as exc:            # capture refused: keep the eager number
             launch_mode = f"eager launches (graph capture failed: {type(exc).__name__})"
+    # node shards: `by` is the whole job's; value shards: `by` is this rank's 1/world of the job
     value = whole_job_value(1 if sharded else world, by["iv_read"], ms_per_step)
 
     # ---- end to end through the host-buffer entry point ------------------
@@ -430,7 +470,7 @@ def run_ours(args, w):
     try:
         if args.skip_e2e:
             raise RuntimeError("--skip-e2e")
-        if sharded:
+        if sharded or value_sharded:
             raise RuntimeError("host-buffer leg is defined for the unsharded workloads")
         import psutil
 
@@ -523,13 +563,16 @@ def run_ours(args, w):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
-        "scaling": "strong" if sharded else "weak",
+        "scaling": "strong" if (sharded or value_sharded) else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w.name, "parallelism": f"nodes sharded over {world} GPUs, all-gather of coded rows" if sharded
+        "config": {"workload": w.name, "parallelism": f"nodes sharded over {world} GPUs, {wire['exchange']}" if sharded
+                   else f"one job, every segment cut into {world} sub-ranges, one per GPU, no exchange (B={full_B})" if value_sharded
                    else f"{world} independent job(s), one per GPU", "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,
+                   **({"wire": wire} if wire else {}),
                    "l2": (f"inputs ({input_bytes / 1e9:.1f} GB) larger than L2, no flush" if flush is None else
                           f"inputs ({input_bytes / 1e9:.3f} GB) fit in L2: 512 MB written, then 512 MB read, between steps; steps timed one by one"),
                    "step": "Map + shuffle (job time)" if w.map_rows else "shuffle", "jobs_per_gpu": plan.J,
+                   "kernels": {"encode": ccdc.last_gather_kernel(), "decode": ccdc.last_decode_kernel()},
                    "launch": launch_mode, **({"eager_ms_per_step": eager_ms} if launch_mode.startswith("one") else {}),
                    **({"map_kernel": ccdc.map_last_kernel()} if w.map_rows else {}),
                    "load_per_JQT": plan.coded_bits / (plan.J * w.Q * 32 * w.B),
@@ -612,6 +655,49 @@ def run_compression(args, w):
     }))
 
 
+def run_load_table(args):
+    """One JSON line per workload: the multicast words the fused encode really wrote (counted on the
+    device: the coded buffer starts full of a mark, the partitions hold zeros, so every word written
+    is a zero), times 32, beside the plan's count and the paper's loads -- Theorem 1, the plain CDC
+    load and the compression-only load of Eq. (2) -- in the paper's normalisation (bits / (J Q T))."""
+    import torch
+    from fractions import Fraction
+    from math import ceil, comb
+
+    from paper_1805_01993_b200 import build as lib_build
+    from paper_1805_01993_b200 import ccdc
+
+    lib_build.build_library()
+    torch.cuda.set_device(0)
+    for name in sorted(CONFIGS):
+        w = CONFIGS[name]
+        plan = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=w.jobs)
+        part = [torch.zeros(plan.partition_bytes(k) // 4, dtype=plan.torch_dtype, device="cuda") for k in range(w.K)]
+        coded = torch.full((plan.coded_bytes // 4,), -0x7A5A5A5B, dtype=torch.int32, device="cuda")
+        plan.encode_fused(part, coded.view(plan.torch_dtype))
+        torch.cuda.synchronize()
+        written = int((coded != -0x7A5A5A5B).sum().item())
+        del part, coded
+        torch.cuda.empty_cache()
+        mu = Fraction(w.r, w.K)
+        T = 32 * w.B
+        # one job over all K nodes carries C(K,r)/(r+1) of the paper's jobs (a paper job has r+1 batches)
+        jobs_eq = Fraction(plan.J) if w.jobs else Fraction(comb(w.K, w.r), w.r + 1)
+        theorem1 = (1 - mu) * (w.r + 1) / w.r
+        length = (w.Q // w.K) * w.B
+        pad = Fraction(w.r * plan.segment_elems, length)      # zero extension when r does not divide the packet
+        print(json.dumps({
+            "workload": name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B, "jobs": plan.J,
+            "coded_bits_counted_on_device": written * 32, "coded_bits_plan": plan.coded_bits,
+            "load_measured": float(Fraction(written * 32) / (jobs_eq * w.Q * T)),
+            "load_theorem1": float(theorem1), "segment_padding_factor": float(pad),
+            "measured_over_theorem1": float(Fraction(written * 32) / (jobs_eq * w.Q * T) / theorem1),
+            # plain CDC on a paper job of r+1 batches of b files, (1-mu) N / (mu K) with N = (r+1) b: no combining
+            "load_cdc": float(theorem1 * plan.files_per_batch),
+            "load_compression_eq2": float(ceil(1 / mu) - 1 if mu < Fraction(1, 2) else 1),
+            "normalisation": "bits / (J Q T); a single job over all K nodes counts as C(K,r)/(r+1) jobs"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -625,13 +711,25 @@ def main():
                     help="compression = the appendix's compression-only shuffle, as a comparator")
     ap.add_argument("--shard-nodes", action="store_true",
                     help="with N > 1 GPUs: one job, K/N logical nodes per GPU, coded rows all-gathered (strong scaling)")
+    ap.add_argument("--peer-stores", action="store_true",
+                    help="with --shard-nodes: the encode kernel stores its rows into every GPU's coded buffer (peer mappings) "
+                         "instead of an all-gather")
+    ap.add_argument("--shard-values", action="store_true",
+                    help="with N > 1 GPUs: one job, every GPU owns one sub-range of every segment, no exchange (strong scaling)")
+    ap.add_argument("--load-table", action="store_true",
+                    help="print, per workload, the multicast bits counted on the device against the paper's loads, and exit")
+    ap.add_argument("--family", type=int, choices=[0, 1], default=None,
+                    help="kernel family override: 0 = loads through registers, 1 = bulk-copy pipelines (default: the planner's choice)")
+    ap.add_argument("--decode-chunks", type=int, default=0, help="override the split of the fused decode's batch loop")
     ap.add_argument("--skip-e2e", action="store_true", help="leave out the host-buffer leg")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="leave out the oracle timing leg")
     args = ap.parse_args()
     w = CONFIGS[args.workload]
     if args.value_elems:
         w = w.scaled(args.value_elems)
-    if args.impl == "reference":
+    if args.load_table:
+        run_load_table(args)
+    elif args.impl == "reference":
         run_reference(args, w)
     elif args.scheme == "compression":
         run_compression(args, w)

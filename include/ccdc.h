@@ -158,6 +158,20 @@ int  ccdc_plan_upload(ccdc_plan_t *plan);
  * 512 or 1024 (CCDC_EINVAL otherwise); only before the tables are uploaded
  * (CCDC_ESTATE after).  Results do not depend on the shape for int32; for fp32
  * the grouping of the per-batch terms follows the chunks (Eq. (1) is a sum). */
+/* Kernel family of the fused encode and decode: 0 = loads through registers
+ * (any plan), 1 = bulk-copy pipelines: one thread per block streams whole
+ * operand rows into a ring of shared-memory stages with asynchronous bulk
+ * copies and the other threads fold them (needs 4 | (Q/K)*B, 2 | s and a
+ * device of compute capability >= 9; CCDC_ESIZE otherwise).  The planner
+ * chooses; ccdc_plan_tune_family overrides, before the tables are uploaded
+ * (CCDC_ESTATE after), and re-sizes the split of the decode for the family.
+ * Both families add in the same order and give the same bits.  The waits of
+ * family 1 are bounded; ccdc_shuffle_status (call it after synchronising the
+ * stream; copies one word back) returns CCDC_ESTATE if one ever ran out on
+ * this plan, in which case that call's outputs are not valid. */
+int  ccdc_plan_kernel_family(const ccdc_plan_t *plan);
+int  ccdc_plan_tune_family(ccdc_plan_t *plan, int family);
+int  ccdc_shuffle_status(const ccdc_plan_t *plan);
 int  ccdc_plan_decode_threads(const ccdc_plan_t *plan);
 int  ccdc_plan_decode_chunks(const ccdc_plan_t *plan);
 int  ccdc_plan_tune_decode(ccdc_plan_t *plan, int threads, int chunks);

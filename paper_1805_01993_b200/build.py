@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libccdc.so"
-SOURCES = ["ccdc_plan.cpp", "ccdc_kernels.cu", "ccdc_map.cu", "ccdc_map_cluster.cu", "ccdc_multi.cu"]
+SOURCES = ["ccdc_plan.cpp", "ccdc_kernels.cu", "ccdc_map.cu", "ccdc_map_cluster.cu", "ccdc_multi.cu", "ccdc_stream.cu"]
 
 
 def nvcc_command(out: Path, verbose: bool = False, defines: tuple[str, ...] = ()) -> list[str]:

@@ -35,6 +35,9 @@ SIGNATURES = {
     "ccdc_coded_send_bytes": (_SZ, [_P]),
     "ccdc_plan_destroy": (None, [_P]),
     "ccdc_plan_upload": (_I, [_P]),
+    "ccdc_plan_kernel_family": (_I, [_P]),
+    "ccdc_plan_tune_family": (_I, [_P, _I]),
+    "ccdc_shuffle_status": (_I, [_P]),
     "ccdc_plan_decode_threads": (_I, [_P]),
     "ccdc_plan_decode_chunks": (_I, [_P]),
     "ccdc_plan_tune_decode": (_I, [_P, _I, _I]),
@@ -272,6 +275,18 @@ class Plan:
 
     def coded_row_position(self, g, a):
         return lib().ccdc_plan_coded_row_position(self._h, g, a)
+
+    @property
+    def kernel_family(self):
+        return lib().ccdc_plan_kernel_family(self._h)
+
+    def tune_family(self, family):
+        """0: loads through registers; 1: bulk-copy pipelines (before the tables are uploaded)."""
+        _check(lib().ccdc_plan_tune_family(self._h, family), "ccdc_plan_tune_family")
+
+    def shuffle_status(self):
+        """after a synchronise: raises if a bounded wait inside a kernel ever ran out on this plan."""
+        _check(lib().ccdc_shuffle_status(self._h), "ccdc_shuffle_status")
 
     @property
     def decode_threads(self):

@@ -24,11 +24,20 @@
 #ifndef CCDC_DECODE_GROUP_WORDS
 #define CCDC_DECODE_GROUP_WORDS 40      // most words per thread a batch may keep in flight
 #endif
+#ifndef CCDC_STREAM_TILE_WORDS
+#define CCDC_STREAM_TILE_WORDS 2048     // bulk-copy pipeline: words of a segment per block (a multiple of 512)
+#endif
+#ifndef CCDC_STREAM_SMEM_BYTES
+#define CCDC_STREAM_SMEM_BYTES (72 * 1024)  // bulk-copy pipeline: shared memory per block (three blocks per SM)
+#endif
 #ifndef CCDC_DECODE_VECTORS
 #define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
 #ifndef CCDC_DECODE_DEPTH
 #define CCDC_DECODE_DEPTH 2         // batches whose loads are issued together (one-file batches, r <= 4)
+#endif
+#ifndef CCDC_DECODE_DEPTH_FILES
+#define CCDC_DECODE_DEPTH_FILES 3   // the same when several files of a batch are loaded together
 #endif
 #ifndef CCDC_GATHER_THREADS
 #define CCDC_GATHER_THREADS 128
@@ -72,6 +81,37 @@ struct ccdc_gather_table {
     // device copies
     const ccdc_row *d_rows = nullptr;
     const ccdc_ref *d_refs = nullptr;
+};
+
+// Bulk-copy pipeline (ccdc_stream.cu): the source rows of an output segment
+// (decode) or of a coded row (encode), flattened.  A "cell" is one output
+// segment / coded row; its rows are listed in the order they are folded.
+enum {
+    CCDC_SROW_FIRST_FILE = 1,   // first file of an operand: starts the file sum
+    CCDC_SROW_LAST_FILE = 2,    // last file of an operand: the sum enters the batch's XOR
+    CCDC_SROW_CODED = 4,        // a coded packet: starts the batch's XOR as it is
+    CCDC_SROW_FIRST_OP = 8,     // first operand of a batch
+    CCDC_SROW_LAST_OP = 16,     // last operand of a batch: the XOR is added to the output
+    CCDC_SROW_FROM_CODED = 32   // the row is read from the coded buffer, not from the node's partition
+};
+struct ccdc_stream_row {
+    long long off;      // word offset of the segment in its buffer
+    int vl;             // leading words of the segment that exist
+    int flags;
+};
+struct ccdc_stream_cell {
+    long long row0;     // first entry of the cell in the row list
+    long long dst_off;  // word offset of the cell's output
+    int src_node;       // whose partition the rows are read from
+    int seglen;         // words of the output
+};
+struct ccdc_stream_table {
+    std::vector<ccdc_stream_row> rows;
+    std::vector<ccdc_stream_cell> cells;
+    std::vector<int> chunk_row0;        // [cells][nchunk + 1]: first row of each chunk of the batch loop, cell relative
+    const ccdc_stream_row *d_rows = nullptr;
+    const ccdc_stream_cell *d_cells = nullptr;
+    const int *d_chunk_row0 = nullptr;
 };
 
 struct ccdc_plan_s {
@@ -125,12 +165,21 @@ struct ccdc_plan_s {
     const ccdc_ref *d_red_terms = nullptr;
 
     int sm_count = 148;       // SMs the launch shapes are sized for (the device's count once uploaded)
+    int family = 0;           // 0: loads through registers; 1: bulk-copy pipelines (ccdc_stream.cu)
+    bool family_tuned = false;
+    int device_has_bulk_copies = 1;     // compute capability >= 9.0 (known once uploaded)
+    int *d_status = nullptr;  // one word, set by a kernel whose bounded wait ran out
+    ccdc_stream_table enc_stream, dec_stream;   // built at upload for family 1
     int device = -1;          // device holding the table copies, -1 = none
     void *d_blob = nullptr;   // one allocation for all of them
 };
 
 // implemented in ccdc_plan.cpp: sizes the split of the fused decode again for a device with sm_count SMs
 void ccdc_internal_resplit(ccdc_plan_s *plan, int sm_count);
+// implemented in ccdc_plan.cpp: the row lists of the bulk-copy pipeline for the plan's final split
+void ccdc_internal_build_stream_tables(ccdc_plan_s *plan);
+// implemented in ccdc_plan.cpp: the split for the plan's current kernel family
+void ccdc_internal_choose_split(ccdc_plan_s *plan);
 // implemented in ccdc_kernels.cu
 void ccdc_internal_release_device(ccdc_plan_s *plan);
 int ccdc_internal_cuda_fail(int cuda_error);    // records the error for ccdc_last_cuda_error; returns CCDC_ECUDA

@@ -29,6 +29,7 @@
 #include <utility>
 
 #include "ccdc_internal.h"
+#include "ccdc_stream.h"
 
 namespace {
 
@@ -322,9 +323,13 @@ k_gather(const __grid_constant__ GatherParams p) {
 #define CCDC_GATHER_FILES_VECTORS 2       // vectors per thread per tile when several files are loaded together
 #endif
 #ifndef CCDC_GATHER_GROUP_WORDS
-#define CCDC_GATHER_GROUP_WORDS 48        // most words per thread a group of files may keep in flight
+#define CCDC_GATHER_GROUP_WORDS 24        // most words per thread a group of files may keep in flight
+#endif
+#ifndef CCDC_GATHER_FILES_THREADS
+#define CCDC_GATHER_FILES_THREADS 128     // threads per block when several files are loaded together
 #endif
 constexpr int STHREADS = CCDC_STATIC_GATHER_THREADS;
+constexpr int FTHREADS = CCDC_GATHER_FILES_THREADS;
 constexpr int FSU = CCDC_GATHER_FILES_VECTORS;
 
 template <int VEC, bool F32, int RS, int G, int SU, int NT>
@@ -490,7 +495,7 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
         }
         if constexpr (R1S >= 0) {
             constexpr int NSLOT = (1 + R1S * G) > G ? (1 + R1S * G) : G;     // vectors a batch keeps in flight
-            constexpr int DEPTH = NSLOT * VEC * DUNROLL <= 18 ? CCDC_DECODE_DEPTH : 1;
+            constexpr int DEPTH = NSLOT * VEC * DUNROLL <= 18 ? (G > 1 ? CCDC_DECODE_DEPTH_FILES : CCDC_DECODE_DEPTH) : 1;
             const int nb = G == 1 ? 1 : p.b;
             for (int t = 0; t < nt; t += DEPTH) {
                 Words<VEC> v[DEPTH][NSLOT][DUNROLL];
@@ -744,7 +749,7 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
         while (group > 2 && T.na * group * VEC * FSU > CCDC_GATHER_GROUP_WORDS) group /= 2;
         // long one-file rows (the gradient-sized workload): 512-thread blocks measured 2 % faster; short rows lose with them
         const bool wide = lean && group == 1 && T.n_max >= (long long)CCDC_GATHER_WIDE_ROW;
-        const int sthreads = wide ? 2 * STHREADS : STHREADS;
+        const int sthreads = wide ? 2 * STHREADS : group > 1 ? FTHREADS : STHREADS;
         const int svectors = group == 1 ? 2 : FSU;          // vectors per thread per tile
         const long long tile = lean ? (long long)sthreads * VEC * svectors : (long long)GTHREADS * VEC * GUNROLL;
         // a block covers up to 32 tiles of a row, fewer while that would
@@ -760,8 +765,8 @@ int launch_gather(const ccdc_plan_s &P, const ccdc_gather_table &T, const void *
                 constexpr int RS = decltype(rs)::value;
                 if (wide) launch_kernel(k_gather_static<VEC, F32, RS, 1, 2, 2 * STHREADS>, blocks, 2 * STHREADS, 0, st, gp);
                 else if (group == 1) launch_kernel(k_gather_static<VEC, F32, RS, 1, 2, STHREADS>, blocks, STHREADS, 0, st, gp);
-                else if (group == 2) launch_kernel(k_gather_static<VEC, F32, RS, 2, FSU, STHREADS>, blocks, STHREADS, 0, st, gp);
-                else launch_kernel(k_gather_static<VEC, F32, RS, 4, FSU, STHREADS>, blocks, STHREADS, 0, st, gp);
+                else if (group == 2) launch_kernel(k_gather_static<VEC, F32, RS, 2, FSU, FTHREADS>, blocks, FTHREADS, 0, st, gp);
+                else launch_kernel(k_gather_static<VEC, F32, RS, 4, FSU, FTHREADS>, blocks, FTHREADS, 0, st, gp);
             };
             switch (T.na) {
             case 1: go(std::integral_constant<int, 1>()); break;
@@ -825,10 +830,18 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return cuda_fail(e);
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    plan->device_has_bulk_copies = major >= 9;
+    if (plan->family == 1 && !ccdc_stream_supported(*plan)) {      // a device without bulk copies
+        plan->family = 0;
+        ccdc_internal_choose_split(plan);
+    }
     ccdc_internal_resplit(plan, sms);       // launch shapes for this device's SM count
     struct Piece { const void *src; size_t bytes; const void **dst; };
     ccdc_gather_table *tabs[4] = {&plan->enc_fused, &plan->cmb, &plan->enc_pk, &plan->dec_pk};
-    Piece pieces[11];
+    Piece pieces[18];
     int np = 0;
     for (ccdc_gather_table *T : tabs) {
         pieces[np++] = {T->rows.data(), T->rows.size() * sizeof(ccdc_row), (const void **)&T->d_rows};
@@ -837,6 +850,16 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     pieces[np++] = {plan->dec_terms.data(), plan->dec_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_dec_terms};
     pieces[np++] = {plan->red_terms.data(), plan->red_terms.size() * sizeof(ccdc_ref), (const void **)&plan->d_red_terms};
     pieces[np++] = {plan->out_rows.data(), plan->out_rows.size() * sizeof(int), (const void **)&plan->d_out_rows};
+    if (plan->family == 1) {                    // the row lists of the bulk-copy pipeline, for the final split
+        ccdc_internal_build_stream_tables(plan);
+        for (ccdc_stream_table *S : {&plan->dec_stream, &plan->enc_stream}) {
+            pieces[np++] = {S->rows.data(), S->rows.size() * sizeof(ccdc_stream_row), (const void **)&S->d_rows};
+            pieces[np++] = {S->cells.data(), S->cells.size() * sizeof(ccdc_stream_cell), (const void **)&S->d_cells};
+            pieces[np++] = {S->chunk_row0.data(), S->chunk_row0.size() * sizeof(int), (const void **)&S->d_chunk_row0};
+        }
+    }
+    static const int zero_status = 0;           // the word a kernel sets when a bounded wait runs out
+    pieces[np++] = {&zero_status, sizeof(int), (const void **)&plan->d_status};
     size_t total = 0;
     for (int i = 0; i < np; ++i) total += (pieces[i].bytes + 255) / 256 * 256;
     void *blob = nullptr;
@@ -930,6 +953,10 @@ int ccdc_encode_fused(ccdc_plan_t *plan, const void *const *part, void *coded, v
     int rc = check_ptr_array(*plan, part, has_part);
     if (rc == CCDC_OK) rc = ensure_device(plan);
     if (rc != CCDC_OK) return rc;
+    if (plan->family == 1) {
+        std::snprintf(g_last_gather, sizeof(g_last_gather), "k_stream<encode,tile=%lld>", ccdc_stream_tile_words());
+        return ccdc_stream_encode(*plan, part, coded, static_cast<cudaStream_t>(stream));
+    }
     return launch_gather(*plan, plan->enc_fused, part, nullptr, coded, nullptr, (int)plan->b, plan->row_elems,
                          static_cast<cudaStream_t>(stream));
 }
@@ -971,6 +998,23 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
     dp.nlist = P.shard_world > 1 ? (long long)P.out_rows.size() : dp.nout;
     dp.nterm = P.nterm; dp.terms_per_chunk = P.terms_per_chunk;
     dp.K = P.K; dp.r = P.r; dp.b = (int)P.b; dp.TS = P.term_stride; dp.nchunk = P.nchunk;
+    if (P.family == 1) {
+        std::snprintf(g_last_decode, sizeof(g_last_decode), "k_stream<decode,tile=%lld,chunks=%d>", ccdc_stream_tile_words(),
+                      P.nchunk);
+        rc = ccdc_stream_decode(P, part, coded, out, workspace, st);
+        if (rc != CCDC_OK || P.nchunk == 1) return rc;
+        const long long n = P.J * P.K * P.len;
+        const long long todo = (P.shard_world > 1 ? (long long)P.out_rows.size() : P.J * P.K) * P.len;
+        if (P.dtype == CCDC_F32)
+            launch_kernel(k_sum_chunks<true>, (todo + DTHREADS - 1) / DTHREADS, DTHREADS, 0, st, (const uint32_t *)workspace,
+                          static_cast<uint32_t *>(out), P.shard_world > 1 ? P.d_out_rows : (const int *)nullptr,
+                          P.shard_world > 1 ? (long long)P.out_rows.size() : P.J * P.K, P.len, n, P.nchunk);
+        else
+            launch_kernel(k_sum_chunks<false>, (todo + DTHREADS - 1) / DTHREADS, DTHREADS, 0, st, (const uint32_t *)workspace,
+                          static_cast<uint32_t *>(out), P.shard_world > 1 ? P.d_out_rows : (const int *)nullptr,
+                          P.shard_world > 1 ? (long long)P.out_rows.size() : P.J * P.K, P.len, n, P.nchunk);
+        return check_launch();
+    }
     const int stage_refs = 1024;                                    // 16 KiB of shared memory
     dp.stage_terms = (int)std::max(1LL, std::min<long long>(stage_refs / P.term_stride, P.terms_per_chunk));
     return dispatch(P, [&](auto vec, auto f32) -> int {
@@ -1029,6 +1073,15 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
                (const uint32_t *)dp.ws, dp.out, dp.out_rows, dp.nlist, P.len, n, P.nchunk);
         return check_launch();
     });
+}
+
+int ccdc_shuffle_status(const ccdc_plan_t *plan) {
+    if (!plan) return CCDC_EINVAL;
+    if (!plan->d_status) return CCDC_OK;            // nothing has run yet
+    int word = 0;
+    const cudaError_t e = cudaMemcpy(&word, plan->d_status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return word == 0 ? CCDC_OK : CCDC_ESTATE;
 }
 
 int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *out, void *workspace,

@@ -8,6 +8,7 @@
 #include <new>
 
 #include "ccdc_internal.h"
+#include "ccdc_stream.h"
 
 namespace {
 
@@ -92,7 +93,8 @@ int check_parameters(int K, int r, long long N, int Q, long long B, int dtype) {
 // over blocks.  P.sm_count is 148 (B200) until the tables are uploaded, when
 // the device's own count replaces it.
 long long decode_tiles_per_seg(const ccdc_plan_s &P, int threads) {
-    const long long tile = (long long)threads * P.vec * CCDC_DECODE_VECTORS;
+    // the bulk-copy pipeline covers a fixed number of words per block, whatever the vector width
+    const long long tile = P.family == 1 ? CCDC_STREAM_TILE_WORDS : (long long)threads * P.vec * CCDC_DECODE_VECTORS;
     return (P.s + tile - 1) / tile;
 }
 
@@ -114,7 +116,10 @@ void choose_split(ccdc_plan_s &P, long long nout) {
     // several files per batch: many registers per thread, so small blocks
     P.decode_threads = group > 1 ? CCDC_DECODE_THREADS_FILES : CCDC_DECODE_THREADS;
     // blocks resident per SM at the registers these kernels take
-    auto resident = [&](int threads) { return (long long)P.sm_count * (threads >= 1024 ? 1 : threads >= 512 ? 3 : 768 / threads); };
+    auto resident = [&](int threads) {
+        if (P.family == 1) return (long long)P.sm_count * 3;       // bulk-copy pipeline: shared memory for three blocks
+        return (long long)P.sm_count * (threads >= 1024 ? 1 : threads >= 512 ? 3 : 768 / threads);
+    };
     // enough thread blocks to fill the GPU (8 per SM) while a block still walks a fair number of batches
     auto many_blocks = [&](int threads) {
         const long long base = std::max(1LL, nout * P.r * decode_tiles_per_seg(P, threads));
@@ -140,7 +145,7 @@ void choose_split(ccdc_plan_s &P, long long nout) {
     // short segments of one-file batches: one large block per segment instead of two smaller ones, but only
     // when the launch still has many waves of them (one such block is resident per SM); measured: K=16, r=4
     // gains 0.6 %, K=10, r=3 with 450 blocks would lose 17 %
-    if (group <= 1 && P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
+    if (P.family == 0 && group <= 1 && P.s <= (long long)CCDC_DECODE_THREADS_SHORT * P.vec * CCDC_DECODE_VECTORS &&
         P.s > (long long)CCDC_DECODE_THREADS * P.vec * CCDC_DECODE_VECTORS) {
         const long long n = many_blocks(CCDC_DECODE_THREADS_SHORT);
         const long long per = (P.nterm + n - 1) / n, real = (P.nterm + per - 1) / per;
@@ -542,6 +547,64 @@ int make_compression_plan(int K, int r, long long N, int Q, long long B, ccdc_dt
 
 }  // namespace
 
+void ccdc_internal_build_stream_tables(ccdc_plan_s *plan) {
+    ccdc_plan_s &P = *plan;
+    const int r = P.r, r1 = r - 1, TS = P.term_stride;
+    const long long nb = P.b;
+    // ---- decode: per output segment (out row, segment i) the rows of every batch, ascending
+    ccdc_stream_table &D = P.dec_stream;
+    D.rows.clear(); D.cells.clear(); D.chunk_row0.clear();
+    const long long nout = P.J * P.K;
+    for (long long orow = 0; orow < nout; ++orow)
+        for (int i = 0; i < r; ++i) {
+            const int seglen = (int)seg_valid(P, i);
+            ccdc_stream_cell C = {(long long)D.rows.size(), orow * P.len + (long long)i * P.s, (int)(orow % P.K), seglen};
+            for (long long tt = 0; tt < P.nterm; ++tt) {
+                if (tt % P.terms_per_chunk == 0) D.chunk_row0.push_back((int)((long long)D.rows.size() - C.row0));
+                const ccdc_ref *e = &P.dec_terms[(((size_t)orow * r + i) * P.nterm + tt) * TS];
+                if (e[0].off < 0) {                         // a batch stored at the node: its files
+                    for (long long f = 0; f < nb; ++f)
+                        D.rows.push_back({e[1].off + f * P.row_elems, seglen,
+                                          CCDC_SROW_FIRST_OP | CCDC_SROW_LAST_OP | (f == 0 ? CCDC_SROW_FIRST_FILE : 0) |
+                                              (f == nb - 1 ? CCDC_SROW_LAST_FILE : 0)});
+                    continue;
+                }
+                D.rows.push_back({e[0].off, seglen,
+                                  CCDC_SROW_FROM_CODED | CCDC_SROW_CODED | CCDC_SROW_FIRST_OP | CCDC_SROW_FIRST_FILE |
+                                      CCDC_SROW_LAST_FILE | (r1 == 0 ? CCDC_SROW_LAST_OP : 0)});
+                for (int c = 1; c <= r1; ++c)
+                    for (long long f = 0; f < nb; ++f)
+                        D.rows.push_back({e[c].vl > 0 ? e[c].off + f * P.row_elems : 0, (int)std::min<long long>(seglen, e[c].vl),
+                                          (c == r1 ? CCDC_SROW_LAST_OP : 0) | (f == 0 ? CCDC_SROW_FIRST_FILE : 0) |
+                                              (f == nb - 1 ? CCDC_SROW_LAST_FILE : 0)});
+            }
+            D.chunk_row0.push_back((int)((long long)D.rows.size() - C.row0));
+            D.cells.push_back(C);
+        }
+    // ---- encode: per coded row the files of its r operands
+    ccdc_stream_table &E = P.enc_stream;
+    E.rows.clear(); E.cells.clear(); E.chunk_row0.clear();
+    const ccdc_gather_table &T = P.enc_fused;
+    for (size_t x = 0; x < T.rows.size(); ++x) {
+        const ccdc_row &R = T.rows[x];
+        E.cells.push_back({(long long)E.rows.size(), R.dst_off, R.src_node, (int)R.n});
+        E.chunk_row0.push_back(0);
+        for (int a = 0; a < r; ++a) {
+            const ccdc_ref &ref = T.refs[x * r + a];
+            for (long long f = 0; f < nb; ++f)
+                E.rows.push_back({ref.vl > 0 ? ref.off + f * P.row_elems : 0, (int)std::min(R.n, ref.vl),
+                                  (a == 0 ? CCDC_SROW_FIRST_OP : 0) | (a == r - 1 ? CCDC_SROW_LAST_OP : 0) |
+                                      (f == 0 ? CCDC_SROW_FIRST_FILE : 0) | (f == nb - 1 ? CCDC_SROW_LAST_FILE : 0)});
+        }
+        E.chunk_row0.push_back((int)(r * nb));
+    }
+}
+
+void ccdc_internal_choose_split(ccdc_plan_s *plan) {
+    if (plan->compression_mode || plan->tuned) return;
+    choose_split(*plan, plan->shard_world > 1 ? (long long)plan->out_rows.size() : plan->J * plan->K);
+}
+
 void ccdc_internal_resplit(ccdc_plan_s *plan, int sm_count) {
     if (sm_count < 1 || sm_count == plan->sm_count) return;
     plan->sm_count = sm_count;
@@ -616,6 +679,23 @@ int ccdc_plan_tune_decode(ccdc_plan_t *p, int threads, int chunks) {
     p->decode_threads = threads;
     set_split(*p, chunks);
     p->tuned = true;
+    return CCDC_OK;
+}
+
+int ccdc_plan_kernel_family(const ccdc_plan_t *p) { return p ? p->family : 0; }
+
+int ccdc_plan_tune_family(ccdc_plan_t *p, int family) {
+    if (!p || (family != 0 && family != 1)) return CCDC_EINVAL;
+    if (p->compression_mode || p->device != -1) return CCDC_ESTATE;
+    const int before = p->family;
+    p->family = family;
+    ccdc_internal_choose_split(p);                  // the split follows the family's tile
+    if (family == 1 && !ccdc_stream_supported(*p)) {
+        p->family = before;
+        ccdc_internal_choose_split(p);
+        return CCDC_ESIZE;
+    }
+    p->family_tuned = true;
     return CCDC_OK;
 }
 

@@ -61,8 +61,10 @@ def assert_outputs(out_gpu, o, dtype):
     assert np.all(np.abs(got - s64) <= FP32_RTOL * a64 + 1e-30)
 
 
-def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0, tune=None):
+def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0, tune=None, family=None):
     plan = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+    if family is not None:
+        plan.tune_family(family)
     if tune:
         plan.tune_decode(*tune)
     o = Oracle(K, r, N, Q, B, dtype, mode="paper" if jobs else "single")
@@ -109,6 +111,7 @@ def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0, tune=None)
     if ws_words == 0:
         assert np.array_equal(bits(out2).reshape(-1, B), o.reduce().view(np.uint32))
     assert plan.coded_bits == o.coded_bits
+    plan.shuffle_status()
     return plan
 
 
@@ -158,6 +161,34 @@ def test_single_job_matches_oracle(ccdc, K, r, N, Q, B, dtype):
 def test_jobs_plan_matches_oracle(ccdc, K, r, N, Q, B, dtype):
     """The scheme as stated for J = C(K, r+1) jobs (stages 1 and 2)."""
     run_case(ccdc, K, r, N, Q, B, dtype, jobs=True, seed=3)
+
+
+def bulk_copy_family_serves(K, r, N, Q, B):
+    length = (Q // K) * B
+    return length % 4 == 0 and (-(-length // r)) % 2 == 0
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", SHAPES + [(10, 3, 480, 10, 4096), (8, 3, 112, 8, 1024), (4, 2, 12, 4, 256),
+                                               (6, 2, 15, 6, 4 * 2048 + 2), (5, 3, 10, 5, 3 * 4098)])
+def test_bulk_copy_family_matches_oracle(ccdc, K, r, N, Q, B, dtype):
+    """The fused encode and decode as bulk-copy pipelines (kernel family 1): same coded words, same
+    outputs; shapes the family cannot serve (rows not 16-byte aligned, odd segments) are refused."""
+    if not bulk_copy_family_serves(K, r, N, Q, B):
+        with pytest.raises(ccdc.CcdcError) as e:
+            ccdc.Plan(K, r, N, Q, B, dtype).tune_family(1)
+        assert e.value.status == ccdc.ESIZE
+        return
+    plan = run_case(ccdc, K, r, N, Q, B, dtype, seed=K + r, family=1)
+    assert plan.kernel_family == 1
+    assert "k_stream<encode" in ccdc.last_gather_kernel() and "k_stream<decode" in ccdc.last_decode_kernel()
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", [(4, 2, 6, 4, 8), (5, 2, 9, 5, 36), (6, 4, 10, 6, 4104), (5, 2, 21, 5, 2060)])
+def test_bulk_copy_family_on_the_jobs_plan(ccdc, K, r, N, Q, B, dtype):
+    plan = run_case(ccdc, K, r, N, Q, B, dtype, jobs=True, seed=5, family=1)
+    assert "k_stream<decode" in ccdc.last_decode_kernel()
 
 
 def test_cfg1_full(ccdc):
