@@ -174,6 +174,11 @@ int  ccdc_plan_tune_family(ccdc_plan_t *plan, int family);
 int  ccdc_shuffle_status(const ccdc_plan_t *plan);
 int  ccdc_plan_decode_threads(const ccdc_plan_t *plan);
 int  ccdc_plan_decode_chunks(const ccdc_plan_t *plan);
+/* 1 if the blocks that share an output tile (one per chunk) form a thread-block cluster and add their
+ * partial sums through distributed shared memory, in chunk order: then ccdc_workspace_bytes is 0 and
+ * ccdc_decode_reduce is a single launch.  Chosen for 2..8 chunks on plans with several files per batch
+ * (r <= 4, even segment length); other split plans use the workspace and a second small launch. */
+int  ccdc_plan_decode_cluster(const ccdc_plan_t *plan);
 int  ccdc_plan_tune_decode(ccdc_plan_t *plan, int threads, int chunks);
 
 /* ---------------------------------------------------------------- queries
@@ -298,8 +303,9 @@ int ccdc_reduce(ccdc_plan_t *plan, const void *const *part, const void *const *d
  *   the batches of the job in ascending order, the local pre-combined word, or
  *   the coded word XOR the r-1 cancellable pre-combined words (decoding of
  *   Section IV-B), accumulated as Eq. (1) demands.  When the loop over the
- *   batches is split over several blocks, each leaves its partial sum in the
- *   workspace and a second small launch adds them in chunk order.  workspace:
+ *   batches is split over several blocks, the partial sums are added in chunk
+ *   order: inside a thread-block cluster (ccdc_plan_decode_cluster), or from
+ *   the workspace by a second small launch.  workspace:
  *   ccdc_workspace_bytes (may be NULL if that is 0); it is fully overwritten
  *   before it is read.  int32 outputs are
  *   bit-identical to the stepwise path; fp32 outputs are too when the

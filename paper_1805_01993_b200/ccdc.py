@@ -40,6 +40,7 @@ SIGNATURES = {
     "ccdc_shuffle_status": (_I, [_P]),
     "ccdc_plan_decode_threads": (_I, [_P]),
     "ccdc_plan_decode_chunks": (_I, [_P]),
+    "ccdc_plan_decode_cluster": (_I, [_P]),
     "ccdc_plan_tune_decode": (_I, [_P, _I, _I]),
     "ccdc_plan_num_jobs": (_LL, [_P]),
     "ccdc_plan_num_batches": (_LL, [_P]),
@@ -295,6 +296,10 @@ class Plan:
     @property
     def decode_chunks(self):
         return lib().ccdc_plan_decode_chunks(self._h)
+
+    @property
+    def decode_cluster(self):
+        return bool(lib().ccdc_plan_decode_cluster(self._h))
 
     def tune_decode(self, threads, chunks):
         """fixes the launch shape of the fused decode (before the tables are uploaded)."""

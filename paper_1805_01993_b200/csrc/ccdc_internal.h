@@ -30,6 +30,9 @@
 #ifndef CCDC_STREAM_SMEM_BYTES
 #define CCDC_STREAM_SMEM_BYTES (72 * 1024)  // bulk-copy pipeline: shared memory per block (three blocks per SM)
 #endif
+#ifndef CCDC_DECODE_CLUSTER_SUM
+#define CCDC_DECODE_CLUSTER_SUM 1       // split batch loop of up to 8 chunks (several files per batch): sum through a cluster
+#endif
 #ifndef CCDC_DECODE_VECTORS
 #define CCDC_DECODE_VECTORS 1       // vectors per thread per tile
 #endif
@@ -136,6 +139,7 @@ struct ccdc_plan_s {
     int term_stride = 0;      // refs per term of the fused decode: 1 + max(r-1, 1)
     int decode_threads = CCDC_DECODE_THREADS;   // block size of the fused decode
     int decode_files = 1;     // files of a batch whose loads the fused decode issues together
+    bool decode_cluster = false;    // the chunks of an output tile meet in a thread-block cluster (no workspace)
     bool tuned = false;       // the caller fixed the decode's launch shape (ccdc_plan_tune_decode)
     int nchunk = 1;           // split of the batch loop in the fused decode
     long long terms_per_chunk = 0;

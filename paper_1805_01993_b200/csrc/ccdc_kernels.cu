@@ -73,19 +73,47 @@ __device__ __forceinline__ void pdl_wait() {
 #endif
 }
 
+// cluster > 1: consecutive groups of `cluster` blocks form a thread-block cluster
 template <typename... KArgs, typename... Args>
-cudaError_t launch_kernel(void (*kernel)(KArgs...), long long grid, int block, size_t smem, cudaStream_t st, Args &&...args) {
+cudaError_t launch_clustered(void (*kernel)(KArgs...), int cluster, long long grid, int block, size_t smem, cudaStream_t st,
+                             Args &&...args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (CCDC_USE_PDL) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = CCDC_USE_PDL ? 1 : 0;
+    cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), long long grid, int block, size_t smem, cudaStream_t st, Args &&...args) {
+    return launch_clustered(kernel, 1, grid, block, smem, st, std::forward<Args>(args)...);
+}
+
+// ---- thread-block clusters: barrier over the blocks of a cluster, loads from a peer block's shared memory
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ unsigned peer_shared_address(const void *local, unsigned rank) {
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"((unsigned)__cvta_generic_to_shared(local)), "r"(rank));
+    return remote;
 }
 
 // ---------------------------------------------------------------- vectors
@@ -111,6 +139,20 @@ __device__ __forceinline__ void store_words(uint32_t *p, const Words<VEC> &x) {
     V v;
     memcpy(&v, x.w, sizeof(V));
     *reinterpret_cast<V *>(p) = v;
+}
+
+// VEC words from the shared memory of block `rank` of this block's cluster, at the slot `local` names here
+template <int VEC>
+__device__ __forceinline__ Words<VEC> load_words_peer(const uint32_t *local, unsigned rank) {
+    const unsigned a = peer_shared_address(local, rank);
+    Words<VEC> out;
+    if constexpr (VEC == 4)
+        asm volatile("ld.shared::cluster.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(out.w[0]), "=r"(out.w[1]), "=r"(out.w[2]), "=r"(out.w[3]) : "r"(a));
+    else if constexpr (VEC == 2)
+        asm volatile("ld.shared::cluster.v2.u32 {%0,%1}, [%2];" : "=r"(out.w[0]), "=r"(out.w[1]) : "r"(a));
+    else
+        asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(out.w[0]) : "r"(a));
+    return out;
 }
 
 template <int VEC>
@@ -445,17 +487,22 @@ constexpr int decode_min_blocks(int vec, int nt, int r1s, int g) {
     return (1 + r1s) * vec * CCDC_DECODE_DEPTH <= 16 ? 3 : 2;
 }
 
-template <int VEC, bool F32, int NT, int R1S, int G>
+// CL: the blocks that share an output tile (one per chunk of the split batch loop) form a thread-block
+// cluster and add their partial sums through distributed shared memory, in chunk order, instead of
+// through the workspace and a second launch.
+template <int VEC, bool F32, int NT, int R1S, int G, bool CL>
 __global__ void __launch_bounds__(NT, decode_min_blocks(VEC, NT, R1S, G))
 k_decode_reduce(const __grid_constant__ DecodeParams p) {
     constexpr long long TILE = (long long)NT * VEC * DUNROLL;
     extern __shared__ ccdc_ref sh_terms[];
 
     long long item = blockIdx.x;
+    int chunk = 0;
+    if constexpr (CL) { chunk = (int)(item % p.nchunk); item /= p.nchunk; }     // the rank in the cluster
     const long long span = item % p.spans_per_seg; item /= p.spans_per_seg;
     const int i = (int)(item % p.r); item /= p.r;
-    const int chunk = (int)(item % p.nchunk);
-    const long long li = item / p.nchunk;
+    if constexpr (!CL) { chunk = (int)(item % p.nchunk); item /= p.nchunk; }
+    const long long li = item;
     if (li >= p.nlist) return;
     const long long orow = p.out_rows ? p.out_rows[li] : li;
 
@@ -599,6 +646,27 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
         }
     }
     const long long cell_off = orow * p.len + (long long)i * p.s;
+    if constexpr (CL) {
+        // every block of the cluster reaches this point for the same tiles (same segment, same span)
+        __shared__ __align__(16) uint32_t sh_part[NT * VEC * DUNROLL];
+#pragma unroll
+        for (int u = 0; u < DUNROLL; ++u) store_words<VEC>(sh_part + (u * NT + (int)threadIdx.x) * VEC, acc[u]);
+        cluster_sync();
+        if (chunk == 0) {
+            for (int c = 1; c < p.nchunk; ++c) {
+#pragma unroll
+                for (int u = 0; u < DUNROLL; ++u)
+                    add_into<VEC, F32>(acc[u], load_words_peer<VEC>(sh_part + (u * NT + (int)threadIdx.x) * VEC, (unsigned)c));
+            }
+#pragma unroll
+            for (int u = 0; u < DUNROLL; ++u) {
+                const long long j = j0 + (long long)u * NT * VEC;
+                if (j < seglen) store_words<VEC>(p.out + cell_off + j, acc[u]);
+            }
+        }
+        cluster_sync();         // a peer's shared memory stays as it is until rank 0 has read it
+        continue;
+    }
     // the output, or this chunk's partial sum when the batch loop is split
     uint32_t *dst = (p.nchunk == 1 ? p.out : p.ws + (long long)chunk * p.nout * p.len) + cell_off;
 #pragma unroll
@@ -646,7 +714,7 @@ struct ReduceParams {
 };
 
 template <int VEC, bool F32>
-__global__ void __launch_bounds__(DTHREADS)
+__global__ void __launch_bounds__(DTHREADS, 2)      // two blocks per SM: up to 64 registers
 k_reduce(const __grid_constant__ ReduceParams p) {
     constexpr long long TILE = (long long)DTHREADS * VEC;
     const long long orow = blockIdx.x / p.tiles_per_row;
@@ -834,6 +902,7 @@ int ccdc_plan_upload(ccdc_plan_t *plan) {
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
     if (e != cudaSuccess) return cuda_fail(e);
     plan->device_has_bulk_copies = major >= 9;
+    if (major < 9) plan->decode_cluster = false;            // no thread-block clusters: the workspace path
     if (plan->family == 1 && !ccdc_stream_supported(*plan)) {      // a device without bulk copies
         plan->family = 0;
         ccdc_internal_choose_split(plan);
@@ -980,10 +1049,11 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
                        void *workspace, void *stream) {
     if (plan && plan->compression_mode) return CCDC_ESTATE;     // no coded path in a compression-only plan
     if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
-    if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
+    if (ccdc_workspace_bytes(plan) > 0 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, part, has_part);
     if (rc == CCDC_OK) rc = ensure_device(plan);
     if (rc != CCDC_OK) return rc;
+    if (ccdc_workspace_bytes(plan) > 0 && !workspace) return CCDC_EINVAL;      // the upload may have re-sized the split
     const ccdc_plan_s &P = *plan;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     DecodeParams dp;
@@ -1042,7 +1112,13 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
             constexpr int NT = decltype(nt)::value;
             constexpr int R1 = decltype(r1)::value;
             constexpr int G = decltype(g)::value;
-            launch_kernel(k_decode_reduce<VEC, F32, NT, R1, G>, blocks, NT, smem, st, dp);
+            if constexpr (G > 1) {
+                if (P.decode_cluster) {
+                    launch_clustered(k_decode_reduce<VEC, F32, NT, R1, G, true>, P.nchunk, blocks, NT, smem, st, dp);
+                    return;
+                }
+            }
+            launch_kernel(k_decode_reduce<VEC, F32, NT, R1, G, false>, blocks, NT, smem, st, dp);
         };
         auto with_shape = [&](auto r1) {
             constexpr int R1 = decltype(r1)::value;
@@ -1064,10 +1140,10 @@ int ccdc_decode_reduce(ccdc_plan_t *plan, const void *const *part, const void *c
         } else {
             with_shape(std::integral_constant<int, -1>());
         }
-        std::snprintf(g_last_decode, sizeof(g_last_decode), "k_decode_reduce<vec=%d,threads=%d,cancel=%d,files=%d,chunks=%d>",
-                      VEC, P.decode_threads, r1s, group, P.nchunk);
+        std::snprintf(g_last_decode, sizeof(g_last_decode), "k_decode_reduce<vec=%d,threads=%d,cancel=%d,files=%d,chunks=%d%s>",
+                      VEC, P.decode_threads, r1s, group, P.nchunk, P.decode_cluster ? ",cluster" : "");
         int lrc = check_launch();
-        if (lrc != CCDC_OK || P.nchunk == 1) return lrc;
+        if (lrc != CCDC_OK || P.nchunk == 1 || P.decode_cluster) return lrc;
         const long long n = dp.nout * P.len, todo = dp.nlist * P.len;
         launch_kernel(k_sum_chunks<F32>, (todo + DTHREADS - 1) / DTHREADS, DTHREADS, 0, st,
                (const uint32_t *)dp.ws, dp.out, dp.out_rows, dp.nlist, P.len, n, P.nchunk);
@@ -1088,7 +1164,7 @@ int ccdc_shuffle(ccdc_plan_t *plan, const void *const *part, void *coded, void *
                  void *stream) {
     if (plan && plan->shard_world > 1) return CCDC_ESTATE;       // the coded rows must be exchanged between the two launches
     if (!plan || !coded || !out || !aligned16(coded) || !aligned16(out)) return CCDC_EINVAL;
-    if (plan->nchunk > 1 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
+    if (ccdc_workspace_bytes(plan) > 0 && (!workspace || !aligned16(workspace))) return CCDC_EINVAL;
     int rc = ccdc_encode_fused(plan, part, coded, stream);
     if (rc != CCDC_OK) return rc;
     return ccdc_decode_reduce(plan, part, coded, out, workspace, stream);
@@ -1113,7 +1189,7 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
                       void *dev_coded, void *dev_out, void *dev_workspace, void *stream) {
     if (!plan || !host_part || !host_out || !dev_part || !dev_coded || !dev_out) return CCDC_EINVAL;
     if (!aligned16(dev_coded) || !aligned16(dev_out)) return CCDC_EINVAL;
-    if (plan->nchunk > 1 && (!dev_workspace || !aligned16(dev_workspace))) return CCDC_EINVAL;
+    if (ccdc_workspace_bytes(plan) > 0 && (!dev_workspace || !aligned16(dev_workspace))) return CCDC_EINVAL;
     int rc = check_ptr_array(*plan, (const void *const *)dev_part, has_part);
     if (rc != CCDC_OK) return rc;
     for (int k = 0; k < plan->K; ++k)

@@ -102,6 +102,10 @@ void set_split(ccdc_plan_s &P, long long nchunk) {
     nchunk = std::max(1LL, std::min(nchunk, P.nterm));
     P.terms_per_chunk = (P.nterm + nchunk - 1) / nchunk;
     P.nchunk = (int)((P.nterm + P.terms_per_chunk - 1) / P.terms_per_chunk);
+    // up to 8 chunks (the portable cluster size) of the kernel form that loads several files together:
+    // the partial sums meet in a thread-block cluster, no workspace
+    P.decode_cluster = CCDC_DECODE_CLUSTER_SUM && P.family == 0 && P.decode_files > 1 && P.nchunk >= 2 && P.nchunk <= 8 &&
+                       P.device_has_bulk_copies;
 }
 
 void choose_split(ccdc_plan_s &P, long long nout) {
@@ -792,8 +796,10 @@ size_t ccdc_coded_bytes(const ccdc_plan_t *p) {
 
 size_t ccdc_out_bytes(const ccdc_plan_t *p) { return p ? (size_t)(p->J * p->row_elems) * 4 : 0; }
 
+int ccdc_plan_decode_cluster(const ccdc_plan_t *p) { return p && p->decode_cluster ? 1 : 0; }
+
 size_t ccdc_workspace_bytes(const ccdc_plan_t *p) {
-    if (!p || p->nchunk <= 1) return 0;
+    if (!p || p->nchunk <= 1 || p->decode_cluster) return 0;
     return (size_t)p->nchunk * (size_t)(p->J * p->row_elems) * 4;
 }
 

@@ -108,7 +108,7 @@ def run_case(ccdc, K, r, N, Q, B, dtype, jobs=False, seed=1, std=1.0, tune=None,
     assert canaries_intact(coded_w2, rows * sp) and canaries_intact(out_w2, plan.J * Q * B)
     assert canaries_intact(ws_w, ws_words)
     assert_outputs(out2, o, dtype)
-    if ws_words == 0:
+    if plan.decode_chunks == 1:          # the batch loop is not split: the oracle's order of additions
         assert np.array_equal(bits(out2).reshape(-1, B), o.reduce().view(np.uint32))
     assert plan.coded_bits == o.coded_bits
     plan.shuffle_status()
@@ -200,7 +200,8 @@ def test_cfg1_full(ccdc):
 def test_cfg2_full(ccdc):
     w = CONFIGS["cfg2"]
     plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype)
-    assert plan.coded_bits == 36_718_080 and plan.workspace_bytes > 0
+    assert plan.coded_bits == 36_718_080 and plan.decode_chunks > 1 and plan.decode_cluster
+    assert "cluster" in ccdc.last_decode_kernel()
 
 
 def test_cfg3_short_values(ccdc):
@@ -244,13 +245,18 @@ def test_cfg5_shuffle_shape(ccdc):
     assert plan.coded_bits == 3_064_320
 
 
-def test_shuffle_replayed_from_a_cuda_graph(ccdc):
+@pytest.mark.parametrize("chunks", [4, 12])
+def test_shuffle_replayed_from_a_cuda_graph(ccdc, chunks):
     """The two launches of ccdc_shuffle (plus the final pass of a split loop) captured in a CUDA graph and
     replayed on new inputs give the oracle's coded packets and outputs: small jobs are launch-bound and
     are meant to be run this way."""
     K, r, N, Q, B, dtype = 10, 3, 480, 10, 96, "float32"          # the K = 10 structure, short values, split loop
     plan = ccdc.Plan(K, r, N, Q, B, dtype)
-    assert plan.workspace_bytes > 0
+    plan.tune_decode(plan.decode_threads, chunks)
+    if chunks > 8:
+        assert plan.workspace_bytes > 0                            # three launches: encode, decode, sum of the partial sums
+    else:
+        assert plan.decode_cluster and plan.workspace_bytes == 0   # two launches, the second one clustered
     part = plan.alloc_partitions()
     coded, out, ws = plan.alloc(plan.coded_bytes), plan.alloc(plan.out_bytes), plan.alloc(plan.workspace_bytes)
     v0 = values_numpy(N, Q, B, dtype, seed=31)
@@ -406,6 +412,7 @@ def test_bad_arguments_are_refused(ccdc):
     with pytest.raises(ccdc.CcdcError):
         plan.shuffle(part, coded[1:], out, None)            # misaligned
     bigplan = ccdc.Plan(10, 3, 480, 10, 64, "int32")
+    bigplan.tune_decode(bigplan.decode_threads, 12)
     assert bigplan.workspace_bytes > 0
     bp = bigplan.alloc_partitions()
     with pytest.raises(ccdc.CcdcError):
@@ -557,7 +564,8 @@ def test_decode_shape_overrides_keep_parity(ccdc, dtype):
             coded = plan.alloc(plan.coded_bytes)
             out_w, out = guarded(Q * B, plan.torch_dtype)
             ws_w, ws = guarded(plan.workspace_bytes // 4, plan.torch_dtype)
-            assert (plan.workspace_bytes > 0) == (chunks > 1)
+            assert (plan.workspace_bytes > 0) == (chunks > 1 and not plan.decode_cluster)
+            assert plan.decode_cluster == (threads == 128 and 2 <= chunks <= 8)
             for _ in range(2):      # the counters of the split loop must be back at zero for the second call
                 plan.shuffle(part, coded, out, ws if plan.workspace_bytes else None)
             torch.cuda.synchronize()

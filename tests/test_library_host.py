@@ -227,11 +227,14 @@ def test_decode_shape_queries_and_override():
     for shape, want in shapes.items():
         p = ccdc.Plan(*shape, "float32")
         assert (p.decode_threads, p.decode_chunks) == want, shape
-        assert (p.workspace_bytes > 0) == (p.decode_chunks > 1)
+        assert (p.workspace_bytes > 0) == (p.decode_chunks > 1) and not p.decode_cluster
     p = ccdc.Plan(10, 3, 480, 10, 4096, "float32")
-    assert p.decode_threads == 128 and 1 < p.decode_chunks <= 15
+    assert p.decode_threads == 128 and 1 < p.decode_chunks <= 8
+    assert p.decode_cluster and p.workspace_bytes == 0      # the chunks meet in a thread-block cluster
     p.tune_decode(128, 6)
-    assert p.decode_chunks == 6 and p.workspace_bytes == 6 * 10 * 4096 * 4
+    assert p.decode_chunks == 6 and p.decode_cluster and p.workspace_bytes == 0
+    p.tune_decode(128, 12)
+    assert p.decode_chunks == 12 and not p.decode_cluster and p.workspace_bytes == 12 * 10 * 4096 * 4
     for threads, chunks in ((256, 6), (128, 0), (128, 121)):
         with pytest.raises(ccdc.CcdcError) as e:
             p.tune_decode(threads, chunks)

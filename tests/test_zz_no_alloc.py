@@ -32,6 +32,7 @@ def ccdc():
 
 def both_ways(ccdc, K, r, N, Q, B, dtype, seed):
     plan = ccdc.Plan(K, r, N, Q, B, dtype)
+    plan.tune_decode(plan.decode_threads, 10)           # a split whose partial sums go through scratch memory
     assert 0 < plan.workspace_bytes <= ccdc.lib().ccdc_static_scratch_bytes()
     plan.upload()
     part = plan.alloc_partitions()
@@ -88,6 +89,7 @@ def test_refuses_what_it_cannot_serve(ccdc):
     assert e.value.status == ccdc.ESIZE
     # tables not on the device yet: uploading them would allocate
     fresh = ccdc.Plan(10, 3, 480, 10, 256, "float32")
+    fresh.tune_decode(fresh.decode_threads, 10)
     with pytest.raises(ccdc.CcdcError) as e:
         fresh.decode_reduce_static([dummy] * 10, dummy, dummy)
     assert e.value.status == ccdc.ESTATE
