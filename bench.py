@@ -41,11 +41,21 @@ UNIT = "GB/s"
 # measured on (hash over the files listed); otherwise the line reports null.
 NCU_TRAFFIC = {
     # workload: (kernel, sources sha256, value elements of the capture, DRAM bytes of that launch, profile)
+    "cfg4": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
+             128000, 3540950008.0, "profiles/ncu_cfg4_small.md"),
+    "cfg3": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
+             8208, 3112038024.0, "profiles/ncu_cfg3_small.md"),
+    "jobs20": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
+             1024, 2256770944.0, "profiles/ncu_jobs20_small.md"),
+    "cfg2": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
+             4096, 143595520.0, "profiles/ncu_cfg2_full.md"),
+    "cfg5": ("k_map", "a7427ce9fd62495f5562f015e6406acaf19ca4a6b7c5b8c4ef81d0fa3406c4a7",
+             1024, 2826514184.0, "profiles/k_map_cluster_cfg5.md"),
 }
 TRAFFIC_SOURCES = {
     "k_decode_reduce": ("ccdc_kernels.cu", "ccdc_internal.h", "ccdc_plan.cpp"),
     "k_gather(encode)": ("ccdc_kernels.cu", "ccdc_internal.h", "ccdc_plan.cpp"),
-    "k_map": ("ccdc_map_cluster.cu", "ccdc_map_cluster.h", "ccdc_internal.h"),
+    "k_map": ("ccdc_map_cluster.cu", "ccdc_map_cluster.h"),
 }
 
 

@@ -42,6 +42,9 @@
 #ifndef CCDC_DECODE_DEPTH_FILES
 #define CCDC_DECODE_DEPTH_FILES 3   // the same when several files of a batch are loaded together
 #endif
+#ifndef CCDC_DECODE_DEPTH_WORDS
+#define CCDC_DECODE_DEPTH_WORDS 20  // a batch of more words per thread than this is not overlapped with the next
+#endif
 #ifndef CCDC_GATHER_THREADS
 #define CCDC_GATHER_THREADS 128
 #endif

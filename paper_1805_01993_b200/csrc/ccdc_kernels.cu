@@ -365,7 +365,7 @@ k_gather(const __grid_constant__ GatherParams p) {
 #define CCDC_GATHER_FILES_VECTORS 2       // vectors per thread per tile when several files are loaded together
 #endif
 #ifndef CCDC_GATHER_GROUP_WORDS
-#define CCDC_GATHER_GROUP_WORDS 24        // most words per thread a group of files may keep in flight
+#define CCDC_GATHER_GROUP_WORDS 32        // most words per thread a group of files may keep in flight
 #endif
 #ifndef CCDC_GATHER_FILES_THREADS
 #define CCDC_GATHER_FILES_THREADS 128     // threads per block when several files are loaded together
@@ -542,7 +542,7 @@ k_decode_reduce(const __grid_constant__ DecodeParams p) {
         }
         if constexpr (R1S >= 0) {
             constexpr int NSLOT = (1 + R1S * G) > G ? (1 + R1S * G) : G;     // vectors a batch keeps in flight
-            constexpr int DEPTH = NSLOT * VEC * DUNROLL <= 18 ? (G > 1 ? CCDC_DECODE_DEPTH_FILES : CCDC_DECODE_DEPTH) : 1;
+            constexpr int DEPTH = NSLOT * VEC * DUNROLL <= CCDC_DECODE_DEPTH_WORDS ? (G > 1 ? CCDC_DECODE_DEPTH_FILES : CCDC_DECODE_DEPTH) : 1;
             const int nb = G == 1 ? 1 : p.b;
             for (int t = 0; t < nt; t += DEPTH) {
                 Words<VEC> v[DEPTH][NSLOT][DUNROLL];
