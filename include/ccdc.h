@@ -356,6 +356,19 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
                       void *const *dev_part, void *dev_coded, void *dev_out, void *dev_workspace,
                       void *stream);
 
+/* The same from Map results that sit in host memory ONCE per file: host_values is
+ * [J*N files][Q][B] in global file order (pinned memory makes the copies
+ * asynchronous).  Every file is copied to the device once, into the partition of
+ * the first node that stores it (Section IV-A placement), and from there, device
+ * to device, into the partitions of the other r-1 nodes that store it -- the
+ * replicas of a file are bit-identical by the scheme's own premise -- so the
+ * host-to-device traffic is N*Q*B words instead of r times that.  Then
+ * ccdc_shuffle and one device-to-host copy of the outputs.  Plans from ccdc_plan,
+ * ccdc_plan_jobs and ccdc_plan_jobs_gamma (CCDC_ESTATE otherwise).  Enqueues on
+ * `stream` (2*r*N small copy calls) and returns without waiting. */
+int ccdc_shuffle_host_files(ccdc_plan_t *plan, const void *host_values, void *host_out, void *const *dev_part,
+                            void *dev_coded, void *dev_out, void *dev_workspace, void *stream);
+
 /* A whole linear-regression job from HOST memory (Section III: Map phase, Shuffle
  * phase, Reduce outputs): copies node k's files host_x[k] ([files][rows][d] bf16),
  * host_y[k] ([files][rows] fp32) and host_w ([d] bf16) into the device staging

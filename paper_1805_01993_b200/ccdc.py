@@ -78,6 +78,7 @@ SIGNATURES = {
     "ccdc_decode_reduce_static": (_I, [_P, _PP, _P, _P, _P]),
     "ccdc_compression_shuffle": (_I, [_P, _PP, _PP, _P, _P]),
     "ccdc_shuffle_host": (_I, [_P, _PP, _P, _PP, _P, _P, _P, _P]),
+    "ccdc_shuffle_host_files": (_I, [_P, _P, _P, _PP, _P, _P, _P, _P]),
     "ccdc_job_host": (_I, [_P, _PP, _PP, _P, _LL, _P, _PP, _PP, _P, _PP, _P, _P, _P, _P, _P]),
     "ccdc_value_shard": (_I, [_I, _I, _I, _LL, _I, _I, ctypes.POINTER(ctypes.c_longlong)]),
     "ccdc_value_shard_position": (_LL, [_I, _I, _I, _LL, _I, _I, _LL]),
@@ -452,6 +453,13 @@ class Plan:
         _check(lib().ccdc_shuffle_host(self._h, _ptr_array(host_part), host_out.data_ptr(), _ptr_array(part),
                                        coded.data_ptr(), out.data_ptr(), ws, _stream_handle(stream)),
                "ccdc_shuffle_host")
+
+    def shuffle_host_files(self, host_values, host_out, part, coded, out, workspace=None, stream=None):
+        """``host_values``: CPU tensor [J*N][Q][B], every file once (pinned for asynchronous copies)."""
+        ws = workspace.data_ptr() if workspace is not None and workspace.numel() else None
+        _check(lib().ccdc_shuffle_host_files(self._h, host_values.data_ptr(), host_out.data_ptr(), _ptr_array(part),
+                                             coded.data_ptr(), out.data_ptr(), ws, _stream_handle(stream)),
+               "ccdc_shuffle_host_files")
 
     def decode_reduce_static(self, part, coded, out, stream=None):
         """``ccdc_decode_reduce`` with the library's built-in scratch: no allocation."""

@@ -524,6 +524,34 @@ def test_shuffle_from_host_buffers(ccdc, K, r, N, Q, B, dtype):
         assert torch.equal(part[k].cpu(), host_part[k])
 
 
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B,jobs", [(4, 2, 12, 4, 300, False), (6, 3, 20, 12, 2049, False), (5, 2, 9, 5, 64, True)])
+def test_shuffle_from_host_files(ccdc, K, r, N, Q, B, jobs, dtype):
+    """ccdc_shuffle_host_files: every file in host memory once; the library places the r replicas
+    (one host-to-device copy per file, device-to-device for the other holders) and shuffles."""
+    plan = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+    o = Oracle(K, r, N, Q, B, dtype, mode="paper" if jobs else "single")
+    v = values_numpy(plan.J * N, Q, B, dtype, seed=78)
+    o.load_values(v)
+    o.shuffle()
+    host_values = torch.from_numpy(v).pin_memory()
+    host_out = torch.full((plan.J * Q * B,), 7, dtype=plan.torch_dtype).pin_memory()
+    part = plan.alloc_partitions()
+    for p_ in part:
+        p_.fill_(3)
+    coded, out = plan.alloc(plan.coded_bytes), plan.alloc(plan.out_bytes)
+    ws = plan.alloc(plan.workspace_bytes)
+    plan.shuffle_host_files(host_values, host_out, part, coded, out, ws if ws.numel() else None)
+    torch.cuda.synchronize()
+    ref_part = plan.alloc_partitions()
+    plan.fill_partitions(ref_part, torch.from_numpy(v).cuda())
+    for k in range(K):
+        assert torch.equal(part[k], ref_part[k]), f"partition of node {k}"
+    s, sp = plan.segment_elems, plan.coded_row_elems
+    assert np.array_equal(bits(coded).reshape(-1, sp)[:, :s], o.coded().reshape(-1, s))
+    assert_outputs(host_out, o, dtype)
+
+
 @pytest.mark.parametrize("K,r,N,Q,B,jobs", [(5, 2, 10, 5, 1000, False), (10, 3, 480, 10, 64, False),
                                             (4, 2, 12, 8, 37, False), (5, 2, 9, 5, 50, True)])
 def test_words_written_by_the_encode_are_the_multicast_bits(ccdc, K, r, N, Q, B, jobs):
