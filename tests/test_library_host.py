@@ -240,3 +240,43 @@ def test_decode_shape_queries_and_override():
             p.tune_decode(threads, chunks)
         assert e.value.status == ccdc.EINVAL
     assert ccdc.last_gather_kernel() == "" or "k_gather" in ccdc.last_gather_kernel()
+
+
+def test_bench_byte_counts_agree_with_the_plan():
+    """The benchmark's algorithmic byte counts against the plan's own sizes, and its DRAM-traffic
+    table: an entry applies only to the kernel sources it was measured on and scales with B."""
+    import sys
+
+    sys.path.insert(0, str(ROOT))
+    import bench
+    from paper_1805_01993_b200.inputs import CONFIGS
+
+    for name in ("cfg1", "cfg2", "cfg3", "cfg4", "cfg5"):
+        w = CONFIGS[name]
+        p = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype)
+        by = bench.algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B)
+        assert by["coded_write"] * 8 == p.coded_bits
+        stored = sum(p.partition_bytes(k) for k in range(w.K))
+        assert stored == w.r * w.N * w.Q * w.B * 4
+        # every node reads, of every stored file, its own function's value and the K-r outside nodes' values
+        assert by["iv_read"] == stored // w.Q * (w.Q // w.K) * (w.K - w.r + 1)
+        assert by["total"] == by["encode_kernel"] + by["decode_kernel"]
+    w = CONFIGS["jobs20"]
+    p = ccdc.Plan(w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=True)
+    by = bench.algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B, J=p.J, rounds=p.num_groups)
+    assert by["coded_write"] * 8 == p.coded_bits
+    assert bench.measured_traffic(CONFIGS["cfg1"], "k_decode_reduce") == (None, None)
+    full, kind = bench.measured_traffic(CONFIGS["cfg4"], "k_decode_reduce")
+    if full is not None:                                    # the table matches the current kernel sources
+        half, _ = bench.measured_traffic(CONFIGS["cfg4"].scaled(640000), "k_decode_reduce")
+        assert "scaled" in kind and half == pytest.approx(full / 2)
+        assert 0.8 < full / by_of("cfg4")["decode_kernel"] < 1.1
+        assert bench.measured_traffic(CONFIGS["cfg4"], "k_gather(encode)") == (None, None)
+
+
+def by_of(name):
+    import bench
+    from paper_1805_01993_b200.inputs import CONFIGS
+
+    w = CONFIGS[name]
+    return bench.algorithmic_bytes(w.K, w.r, w.N, w.Q, w.B)
