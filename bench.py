@@ -41,16 +41,14 @@ UNIT = "GB/s"
 # measured on (hash over the files listed); otherwise the line reports null.
 NCU_TRAFFIC = {
     # workload: (kernel, sources sha256, value elements of the capture, DRAM bytes of that launch, profile)
-    "cfg4": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
-             128000, 3540950008.0, "profiles/ncu_cfg4_small.md"),
-    "cfg3": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
-             8208, 3112038024.0, "profiles/ncu_cfg3_small.md"),
-    "jobs20": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
-             1024, 2256770944.0, "profiles/ncu_jobs20_small.md"),
-    "cfg2": ("k_decode_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
-             4096, 143595520.0, "profiles/ncu_cfg2_full.md"),
-    "compression:cfg4": ("k_gather(combine)+k_reduce", "7945a05ca60a465046256ade8fd5aa8d1fa8f5c65f733ca376e2bd656666299a",
-             128000, 2137791288.0, "profiles/ncu_compression_small.md"),
+    "cfg4": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
+             128000, 3539097792.0, "profiles/ncu_cfg4_small.md"),
+    "cfg3": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
+             8208, 3112820984.0, "profiles/ncu_cfg3_small.md"),
+    "jobs20": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
+             1024, 2256258392.0, "profiles/ncu_jobs20_small.md"),
+    "cfg2": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
+             4096, 143563520.0, "profiles/ncu_cfg2_full.md"),
     "cfg5": ("k_map", "a7427ce9fd62495f5562f015e6406acaf19ca4a6b7c5b8c4ef81d0fa3406c4a7",
              1024, 2826514184.0, "profiles/k_map_cluster_cfg5.md"),
 }

@@ -82,7 +82,8 @@ typedef enum {
  * member t of S receives the batch labelled S\{t}.  Node k reduces functions
  * k*Q/K .. (k+1)*Q/K-1.
  *   requires 2 <= K <= CCDC_MAX_K, 1 <= r <= K-1, K <= N, C(K,r) | N, K | Q,
- *   B >= 1; otherwise CCDC_EINVAL and *out = NULL.
+ *   B >= 1; otherwise CCDC_EINVAL and *out = NULL.  CCDC_ESIZE when the schedule
+ *   is too large to tabulate (more than 2^24 rounds, or decode tables beyond 2 GB).
  *
  * ccdc_plan_jobs: the scheme as Section IV states it for J = C(K,r+1) jobs
  * (gamma = 1).  Job j lives on the j-th size-(r+1) subset K_j; its N files are
@@ -365,7 +366,7 @@ int ccdc_shuffle_host(ccdc_plan_t *plan, const void *const *host_part, void *hos
  * host-to-device traffic is N*Q*B words instead of r times that.  Then
  * ccdc_shuffle and one device-to-host copy of the outputs.  Plans from ccdc_plan,
  * ccdc_plan_jobs and ccdc_plan_jobs_gamma (CCDC_ESTATE otherwise).  Enqueues on
- * `stream` (2*r*N small copy calls) and returns without waiting. */
+ * `stream` (r copy calls per batch of files) and returns without waiting. */
 int ccdc_shuffle_host_files(ccdc_plan_t *plan, const void *host_values, void *host_out, void *const *dev_part,
                             void *dev_coded, void *dev_out, void *dev_workspace, void *stream);
 

@@ -8,16 +8,20 @@
 //
 //   k_gather_static   a destination row = XOR over a compile-time number of
 //                     operands of the batch sums of a segment (the fused encode,
-//                     the stepwise combine and encode); loads in registers
-//   k_gather          the same for any operand count, per-row file counts and
-//                     a coded input row (stepwise decode, compression-only
-//                     unicast); cp.async pipeline through shared memory
+//                     the stepwise combine and encode, the compression-only
+//                     unicast with its per-row file counts); loads in registers
+//   k_gather          the same for any operand count and with a coded input row
+//                     (r > 4, the stepwise decode); cp.async pipeline through
+//                     shared memory
 //   k_decode_reduce   decode + cancel + reduce, decoded packets never stored
 //   k_sum_chunks      ordered sum of the partial outputs when the batch loop
-//                     of k_decode_reduce is split over blocks
+//                     of k_decode_reduce is split over blocks through the workspace
 //   k_reduce          Eq. (1) from materialised packets (stepwise API)
-// No kernel waits on another block or thread: the encode -> decode dependency
-// is the boundary between two launches on one stream.
+// No kernel here spins on memory another block or thread writes: the
+// encode -> decode dependency is the boundary between two launches on one
+// stream (each kernel starts behind griddepcontrol.wait, a dependency the
+// hardware resolves), and the one place blocks meet inside a kernel, the
+// clustered decode, uses the hardware barrier of a thread-block cluster.
 #include <cuda_runtime.h>
 
 #include <atomic>

@@ -90,8 +90,8 @@ int ccdc_value_shard_copy(int K, int r, int Q, long long B, int rank, int world,
 }
 
 // ---- a job whose Map results sit in host memory once per file -------------
-// Every file's Q values are copied to the device once, into the partition of the first node that
-// stores the file, and from there to the other r-1 nodes that store it (device-to-device): the
+// Every batch of files is copied to the device once, into the partition of the first node that
+// stores it, and from there to the other r-1 nodes that store it (device-to-device): the
 // host-to-device traffic is N*Q*B words instead of r times that.
 int ccdc_shuffle_host_files(ccdc_plan_t *plan, const void *host_values, void *host_out, void *const *dev_part,
                             void *dev_coded, void *dev_out, void *dev_workspace, void *stream) {
@@ -101,21 +101,23 @@ int ccdc_shuffle_host_files(ccdc_plan_t *plan, const void *host_values, void *ho
     for (int k = 0; k < P.K; ++k)
         if (P.nlocal[k] > 0 && (!dev_part[k] || (reinterpret_cast<uintptr_t>(dev_part[k]) & 15u))) return CCDC_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const size_t file_bytes = (size_t)P.row_elems * 4;
+    // the files of a batch are consecutive in the host array and in every holder's partition: one copy per
+    // batch and holder
+    const size_t batch_bytes = (size_t)P.b * (size_t)P.row_elems * 4;
     const char *src = static_cast<const char *>(host_values);
-    for (long long p = 0; p < P.nbatch; ++p)
-        for (long long f = 0; f < P.b; ++f) {
-            const long long n = P.batch_file0[p] + f;               // global file id
-            char *first = nullptr;
-            for (int x = 0; x < P.r; ++x) {
-                const int k = P.batch_nodes[(size_t)p * P.r + x];
-                char *dst = static_cast<char *>(dev_part[k]) + (size_t)(P.slot[(size_t)k * P.nbatch + p] * P.b + f) * file_bytes;
-                const cudaError_t e = first ? cudaMemcpyAsync(dst, first, file_bytes, cudaMemcpyDeviceToDevice, st)
-                                            : cudaMemcpyAsync(dst, src + (size_t)n * file_bytes, file_bytes, cudaMemcpyHostToDevice, st);
-                if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
-                if (!first) first = dst;
-            }
+    for (long long p = 0; p < P.nbatch; ++p) {
+        char *first = nullptr;
+        for (int x = 0; x < P.r; ++x) {
+            const int k = P.batch_nodes[(size_t)p * P.r + x];
+            char *dst = static_cast<char *>(dev_part[k]) + (size_t)P.slot[(size_t)k * P.nbatch + p] * batch_bytes;
+            const cudaError_t e =
+                first ? cudaMemcpyAsync(dst, first, batch_bytes, cudaMemcpyDeviceToDevice, st)
+                      : cudaMemcpyAsync(dst, src + (size_t)P.batch_file0[p] * (size_t)P.row_elems * 4, batch_bytes,
+                                        cudaMemcpyHostToDevice, st);
+            if (e != cudaSuccess) return ccdc_internal_cuda_fail((int)e);
+            if (!first) first = dst;
         }
+    }
     const int rc = ccdc_shuffle(plan, (const void *const *)dev_part, dev_coded, dev_out, dev_workspace, stream);
     if (rc != CCDC_OK) return rc;
     const cudaError_t e = cudaMemcpyAsync(host_out, dev_out, ccdc_out_bytes(plan), cudaMemcpyDeviceToHost, st);

@@ -400,6 +400,11 @@ int make_plan(int K, int r, long long N, int Q, long long B, ccdc_dtype_t dtype,
     if (rc != CCDC_OK) return rc;
     const long long n_rsub = choose(K, r), n_r1sub = choose(K, r + 1);
     if (n_rsub <= 0 || n_r1sub <= 0 || n_r1sub > (1LL << 24)) return CCDC_ESIZE;
+    {   // the decode's term table alone: out rows x r segments x batches per job x refs of 16 bytes
+        const long double jobs_n = jobs ? (long double)gamma * n_r1sub : 1.0L;
+        const long double terms = jobs_n * K * r * (jobs ? r + 1 : n_rsub) * (1 + std::max(r - 1, 1)) * 16.0L;
+        if (terms > 2.0e9L) return CCDC_ESIZE;              // host and device tables of more than 2 GB
+    }
     if (!jobs && N % n_rsub != 0) return CCDC_EINVAL;       // batches of equal size
     if (jobs && N % (r + 1) != 0) return CCDC_EINVAL;
     if (gamma < 1 || (!jobs && gamma != 1)) return CCDC_EINVAL;

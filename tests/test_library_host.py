@@ -48,6 +48,9 @@ def test_invalid_parameters():
     with pytest.raises(ccdc.CcdcError) as e:
         ccdc.Plan(32, 15, comb(32, 15), 32, 8, "int32")       # schedule too large
     assert e.value.status == ccdc.ESIZE
+    with pytest.raises(ccdc.CcdcError) as e:
+        ccdc.Plan(20, 10, comb(20, 10), 20, 8, "int32")       # 5.9 GB of decode tables
+    assert e.value.status == ccdc.ESIZE
     assert b"invalid" in ccdc.lib().ccdc_strerror(ccdc.EINVAL)
     assert ccdc.lib().ccdc_plan_num_groups(None) == 0
 
