@@ -608,3 +608,71 @@ def test_decode_shape_overrides_keep_parity(ccdc, dtype):
         with pytest.raises(ccdc.CcdcError) as e:
             bad.tune_decode(threads, chunks)
         assert e.value.status == ccdc.EINVAL
+
+
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+@pytest.mark.parametrize("K,r,N,Q,B", [(3, 1, 30, 3, 2100), (4, 2, 54, 4, 1100), (5, 3, 50, 5, 774), (5, 4, 15, 5, 1304),
+                                       (6, 2, 30, 12, 514)])
+def test_clustered_decode_for_every_operand_count(ccdc, K, r, N, Q, B, dtype):
+    """Splits of 2, 5 and 8 chunks whose partial sums meet in a thread-block cluster, for r = 1..4, 64- and
+    128-bit accesses, ragged tails: outputs against the oracle, no workspace touched."""
+    o = Oracle(K, r, N, Q, B, dtype)
+    v = values_numpy(N, Q, B, dtype, seed=r)
+    o.load_values(v)
+    o.shuffle()
+    for chunks in (2, 5, 8):
+        plan = ccdc.Plan(K, r, N, Q, B, dtype)
+        if chunks > plan.num_batches:
+            continue
+        plan.tune_decode(plan.decode_threads, chunks)
+        assert plan.decode_cluster and plan.workspace_bytes == 0, (K, r, chunks)
+        part = plan.alloc_partitions()
+        plan.fill_partitions(part, torch.from_numpy(v).cuda())
+        coded = plan.alloc(plan.coded_bytes)
+        out_w, out = guarded(Q * B, plan.torch_dtype)
+        plan.shuffle(part, coded, out, None)
+        torch.cuda.synchronize()
+        assert canaries_intact(out_w, Q * B)
+        assert_outputs(out, o, dtype)
+        assert "cluster" in ccdc.last_decode_kernel() and f"chunks={plan.decode_chunks}" in ccdc.last_decode_kernel()
+
+
+@pytest.mark.parametrize("K,r,N,Q,B,chunks", [(6, 2, 15, 6, 3000, 0), (10, 3, 480, 10, 64, 0), (10, 3, 480, 10, 64, 12),
+                                              (8, 4, 70, 8, 4096, 0)])
+def test_back_to_back_steps_on_the_same_buffers(ccdc, K, r, N, Q, B, chunks):
+    """Forty shuffles in a row on one stream without a synchronise, the inputs swapped between two sets
+    before every step: each kernel may be scheduled while its predecessor drains (programmatic dependent
+    launch), so a read or write placed before its dependency wait would show here.  The last two steps'
+    coded rows and outputs are compared with the oracle."""
+    dtype = "int32"
+    plan = ccdc.Plan(K, r, N, Q, B, dtype)
+    if chunks:
+        plan.tune_decode(plan.decode_threads, chunks)
+    sets, refs = [], []
+    for seed in (1, 2):
+        v = values_numpy(N, Q, B, dtype, seed=seed)
+        o = Oracle(K, r, N, Q, B, dtype)
+        o.load_values(v)
+        o.shuffle()
+        refs.append((o.coded().copy(), o.reduce().copy()))
+        p = plan.alloc_partitions()
+        plan.fill_partitions(p, torch.from_numpy(v).cuda())
+        sets.append(p)
+    part = plan.alloc_partitions()
+    coded, out = plan.alloc(plan.coded_bytes), plan.alloc(plan.out_bytes)
+    ws = plan.alloc(plan.workspace_bytes)
+    keep = {}
+    s, sp = plan.segment_elems, plan.coded_row_elems
+    for step in range(40):
+        which = step % 2
+        for dst, src in zip(part, sets[which]):
+            dst.copy_(src, non_blocking=True)
+        plan.shuffle(part, coded, out, ws if ws.numel() else None)
+        if step >= 38:
+            keep[which] = (coded.clone(), out.clone())
+    torch.cuda.synchronize()
+    for which in (0, 1):
+        c, o_ = keep[which]
+        assert np.array_equal(bits(c).reshape(-1, sp)[:, :s], refs[which][0].reshape(-1, s))
+        assert np.array_equal(o_.cpu().numpy().reshape(refs[which][1].shape), refs[which][1])
+    plan.shuffle_status()
