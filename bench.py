@@ -41,14 +41,14 @@ UNIT = "GB/s"
 # measured on (hash over the files listed); otherwise the line reports null.
 NCU_TRAFFIC = {
     # workload: (kernel, sources sha256, value elements of the capture, DRAM bytes of that launch, profile)
-    "cfg4": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
-             128000, 3539097792.0, "profiles/ncu_cfg4_small.md"),
-    "cfg3": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
-             8208, 3112820984.0, "profiles/ncu_cfg3_small.md"),
-    "jobs20": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
-             1024, 2256258392.0, "profiles/ncu_jobs20_small.md"),
-    "cfg2": ("k_decode_reduce", "1e88e2ad3f502934daffaa5c96892813422621f63855173a656cd9fb408cb696",
-             4096, 143563520.0, "profiles/ncu_cfg2_full.md"),
+    "cfg4": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
+             128000, 3542451624.0, "profiles/ncu_cfg4_small.md"),
+    "cfg3": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
+             8208, 3114471640.0, "profiles/ncu_cfg3_small.md"),
+    "jobs20": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
+             1024, 2256828424.0, "profiles/ncu_jobs20_small.md"),
+    "cfg2": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
+             4096, 145249792.0, "profiles/ncu_cfg2_full.md"),
     "cfg5": ("k_map", "a7427ce9fd62495f5562f015e6406acaf19ca4a6b7c5b8c4ef81d0fa3406c4a7",
              1024, 2826514184.0, "profiles/k_map_cluster_cfg5.md"),
 }

@@ -383,18 +383,19 @@ __global__ void __launch_bounds__(NT)
 k_gather_static(const __grid_constant__ GatherParams p) {
     constexpr long long TILE = (long long)NT * VEC * SU;
     const long long item = blockIdx.x;
-    const long long row = item / p.spans_per_row;
-    const long long span = item - row * p.spans_per_row;
-    if (row >= p.nrows) return;
-    const ccdc_row R = p.rows[row];
-    const long long begin = span * p.span_elems;
-    const long long end = min(R.n, begin + p.span_elems);
-    if (begin >= end) return;
+    if (item >= p.nrows * p.spans_per_row) return;
+    // the dependent kernel may be scheduled, and this block's table entries fetched, while the previous
+    // kernel of the stream drains; no data buffer is touched before pdl_wait
     pdl_trigger();
+    const long long row = item / p.spans_per_row;
+    const ccdc_row R = p.rows[row];
     ccdc_ref E[RS];
 #pragma unroll
     for (int a = 0; a < RS; ++a) E[a] = p.refs[row * RS + a];
     pdl_wait();
+    const long long span = item - row * p.spans_per_row;
+    const long long begin = span * p.span_elems;
+    const long long end = min(R.n, begin + p.span_elems);
     const int nb = G == 1 ? 1 : (R.nf > 0 ? (int)R.nf : p.b);      // files summed per operand
     const uint32_t *src = p.src[R.src_node];
     uint32_t *dst = p.dst[p.replicas > 0 ? 0 : R.dst_node] + R.dst_off + p.dst_add;
