@@ -150,35 +150,40 @@ void ccdc_plan_destroy(ccdc_plan_t *plan);
  * there. */
 int  ccdc_plan_upload(ccdc_plan_t *plan);
 
-/* Launch shape of the fused decode (ccdc_decode_reduce), chosen by the planner:
- * threads per block, and the number of blocks (chunks) the loop over a job's
- * batches is split into (1 = no workspace needed).  ccdc_plan_tune_decode
- * overrides the choice, e.g. from a timing sweep; it changes
- * ccdc_workspace_bytes.  Allowed: chunks in 1..batches per job; threads 128 for
- * plans with several files per batch, r <= 4 and an even segment length, else
- * 512 or 1024 (CCDC_EINVAL otherwise); only before the tables are uploaded
- * (CCDC_ESTATE after).  Results do not depend on the shape for int32; for fp32
- * the grouping of the per-batch terms follows the chunks (Eq. (1) is a sum). */
 /* Kernel family of the fused encode and decode: 0 = loads through registers
- * (any plan), 1 = bulk-copy pipelines: one thread per block streams whole
- * operand rows into a ring of shared-memory stages with asynchronous bulk
+ * (any plan; the planner's choice for every plan, it measured faster on every
+ * workload), 1 = bulk-copy pipelines: the lanes of one warp per block stream
+ * whole operand rows into a ring of shared-memory stages with asynchronous bulk
  * copies and the other threads fold them (needs 4 | (Q/K)*B, 2 | s and a
- * device of compute capability >= 9; CCDC_ESIZE otherwise).  The planner
- * chooses; ccdc_plan_tune_family overrides, before the tables are uploaded
- * (CCDC_ESTATE after), and re-sizes the split of the decode for the family.
- * Both families add in the same order and give the same bits.  The waits of
- * family 1 are bounded; ccdc_shuffle_status (call it after synchronising the
- * stream; copies one word back) returns CCDC_ESTATE if one ever ran out on
- * this plan, in which case that call's outputs are not valid. */
+ * device of compute capability >= 9; CCDC_ESIZE otherwise).
+ * ccdc_plan_tune_family selects a family, before the tables are uploaded
+ * (CCDC_ESTATE after), and re-sizes the split of the decode for it.  Both
+ * families add in the same order and give the same bits.  The waits of family 1
+ * are bounded; ccdc_shuffle_status (call it after synchronising the stream;
+ * copies one word back) returns CCDC_ESTATE if one ever ran out on this plan,
+ * in which case that call's outputs are not valid. */
 int  ccdc_plan_kernel_family(const ccdc_plan_t *plan);
 int  ccdc_plan_tune_family(ccdc_plan_t *plan, int family);
 int  ccdc_shuffle_status(const ccdc_plan_t *plan);
+
+/* Launch shape of the fused decode (ccdc_decode_reduce), chosen by the planner:
+ * threads per block, and the number of blocks (chunks) the loop over a job's
+ * batches is split into (1 = no workspace needed).
+ * ccdc_plan_decode_cluster: 1 if the blocks that share an output tile (one per
+ * chunk) form a thread-block cluster and add their partial sums through
+ * distributed shared memory, in chunk order: then ccdc_workspace_bytes is 0 and
+ * ccdc_decode_reduce is a single launch.  Chosen for 2..8 chunks on plans with
+ * several files per batch (r <= 4, even segment length); other split plans use
+ * the workspace and a second small launch.
+ * ccdc_plan_tune_decode overrides the planner's choice, e.g. from a timing
+ * sweep; it changes ccdc_workspace_bytes.  Allowed: chunks in 1..batches per
+ * job; threads 128 for plans with several files per batch, r <= 4 and an even
+ * segment length, else 512 or 1024 (CCDC_EINVAL otherwise); only before the
+ * tables are uploaded (CCDC_ESTATE after).  Results do not depend on the shape
+ * for int32; for fp32 the grouping of the per-batch terms follows the chunks
+ * (Eq. (1) is a sum). */
 int  ccdc_plan_decode_threads(const ccdc_plan_t *plan);
 int  ccdc_plan_decode_chunks(const ccdc_plan_t *plan);
-/* 1 if the blocks that share an output tile (one per chunk) form a thread-block cluster and add their
- * partial sums through distributed shared memory, in chunk order: then ccdc_workspace_bytes is 0 and
- * ccdc_decode_reduce is a single launch.  Chosen for 2..8 chunks on plans with several files per batch
- * (r <= 4, even segment length); other split plans use the workspace and a second small launch. */
 int  ccdc_plan_decode_cluster(const ccdc_plan_t *plan);
 int  ccdc_plan_tune_decode(ccdc_plan_t *plan, int threads, int chunks);
 
