@@ -546,3 +546,34 @@ def test_compression_only_running_example(golden_dir):
     out, recv, bits, files = compression_only(K, r, N, Q, B, "int32", values_numpy(N, Q, B, "int32"))
     assert recv.shape[0] * recv.shape[1] == 4
     assert Fraction(bits, Q * 32 * B) == golden_scalar(rows, "load_compression")
+
+
+@pytest.mark.parametrize("mode", ["single", "paper"])
+@pytest.mark.parametrize("dtype", ["int32", "float32"])
+def test_every_step_acts_word_by_word_along_a_segment(mode, dtype):
+    """Section IV-B: sums, XORs and cancellations combine words at equal positions of equal-size
+    segments only.  So the same sub-range of every segment is itself an instance of the scheme:
+    shuffling the sliced values gives the slices of the coded packets and of the outputs (the property
+    the value-dimension sharding over several GPUs rests on).  Checked on the oracle alone."""
+    K, r, Q, B = 5, 2, 10, 12                   # Q/K = 2: packets of 24 words, segments of 12
+    N = 9 if mode == "paper" else 20
+    per = Q // K
+    full = Oracle(K, r, N, Q, B, dtype, mode=mode)
+    v = values_numpy(full.J * N, Q, B, dtype, seed=17)
+    out = full.run(v)
+    coded = full.coded()                        # [round][sender][s]
+    s = full.s
+    for lo, hi in ((0, 4), (4, 12), (5, 7)):
+        w = hi - lo
+        pos = np.concatenate([np.arange(i * s + lo, i * s + hi) for i in range(r)])
+        assert (r * w) % per == 0
+        b_local = r * w // per
+        packets = v.reshape(full.J * N, K, per * B)
+        local = np.ascontiguousarray(packets[:, :, pos]).reshape(full.J * N, Q, b_local)
+        part = Oracle(K, r, N, Q, b_local, dtype, mode=mode)
+        got = part.run(local)
+        assert part.s == w
+        assert np.array_equal(part.coded(), coded[:, :, lo:hi])
+        want = out.reshape(full.J * K, per * B)[:, pos].reshape(got.shape)
+        assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(want).view(np.uint32))
+        assert part.coded_bits * s == full.coded_bits * w
