@@ -9,10 +9,10 @@
 // that stay: each block walks a contiguous range of output tiles ("items": a
 // tile of a coded row for the encode; a tile of an output segment and one chunk
 // of the job's batches for the decode).  The source rows of all its items form
-// ONE sequence.  The lanes of a producer warp stream that sequence into a ring
-// of shared-memory stages with bulk asynchronous copies (lane l owns stage l),
-// running ahead across item boundaries, so tens of KiB are in flight per block
-// all the time and none of them in registers; 256 consumer threads fold the
+// ONE sequence.  Two producer warps, each owning half of a ring of
+// shared-memory stages (one lane per stage, the lanes in lockstep), stream that
+// sequence in with bulk asynchronous copies, running ahead across item boundaries, so tens of KiB are in flight per block
+// all the time and none of them in registers; 128 consumer threads fold the
 // rows, in the order the scheme fixes, into three registers per word:
 //     S  running sum over the files of the current operand   (pre-combining)
 //     X  XOR over the operands of the current batch           (coding / decoding)
@@ -47,14 +47,15 @@
 
 namespace {
 
-constexpr int CONSUMERS = 256;                  // threads that fold rows
-constexpr int ST_THREADS = CONSUMERS + 32;      // plus the producer warp
+constexpr int CONSUMERS = 128;                  // threads that fold rows
+constexpr int PRODUCERS = 2;                    // producer warps; each owns a contiguous share of the ring's stages
+constexpr int ST_THREADS = CONSUMERS + 32 * PRODUCERS;
 constexpr int TILE_WORDS = CCDC_STREAM_TILE_WORDS;      // words of a segment per item
-constexpr int VECS = TILE_WORDS / (2 * CONSUMERS);      // 64-bit vectors per consumer thread
-constexpr int MAX_STAGES = 32;                  // one producer lane per stage
+constexpr int VECS = TILE_WORDS / (4 * CONSUMERS);      // 128-bit vectors (4 consecutive words) per consumer thread
+constexpr int MAX_STAGES = 32;
 constexpr int WAIT_LIMIT = 1 << 14;             // polls of an mbarrier before giving up (each may sleep up to SLEEP_NS)
 constexpr unsigned SLEEP_NS = 200000;           // time a poll may suspend the thread waiting for the phase to complete
-static_assert(TILE_WORDS % (2 * CONSUMERS) == 0, "tile must be a whole number of vectors per thread");
+static_assert(TILE_WORDS % (4 * CONSUMERS) == 0, "tile must be a whole number of vectors per thread");
 
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count) {
@@ -199,37 +200,58 @@ k_stream(const __grid_constant__ StreamParams p) {
     pdl_wait();
     volatile int *abort_flag = &sh->abort_flag;
 
-    if (warp == CONSUMERS / 32) {
-        // ---------------- producer: lane l brings in rows l, l + nstage, ... of the block's sequence
-        if (lane < p.nstage) {
-            const int st = lane;
+    if (warp >= CONSUMERS / 32) {
+        // ---------------- producers: warp w owns stages [w*G, (w+1)*G), G = nstage / PRODUCERS, lane l of it stage
+        // w*G + l.  Its lanes work in lockstep on one row each (round k: rows k*nstage + stage), so a round
+        // costs one pass of the instruction stream for G rows; the warp refills its stages when all of them
+        // have been released, while the consumers are busy with the other warp's stages.
+        const int pw = warp - CONSUMERS / 32;
+        const int G = p.nstage / PRODUCERS;
+        if (lane < G) {
+            const unsigned mask = G >= 32 ? 0xffffffffu : ((1u << G) - 1u);
+            const int st = pw * G + lane;
             long long it = it0 - 1, first = 0;      // current item and the sequence index of its first row
             int nrows = 0;                          // rows of the current item
             Item I = {0, 0, 0};
             ccdc_stream_cell C = {0, 0, 0, 0};
             long long row_base = 0;
-            unsigned use = 0;                       // how often this lane has filled its stage
             bool ok = true;
-            for (long long n = st; n < total; n += p.nstage, ++use) {
-                while (n >= first + nrows) {        // on to the item that holds row n (items without rows are skipped)
-                    first += nrows;
-                    ++it;
-                    I = item_of(p, it);
-                    nrows = item_rows(p, I);
-                    if (nrows) {
-                        C = p.cells[I.cell];
-                        row_base = C.row0 + p.chunk_row0[I.cell * (p.nchunk + 1) + I.chunk];
+            unsigned round = 0;
+            for (long long n0 = (long long)pw * G; n0 < total && ok; n0 += p.nstage, ++round) {     // n0: the warp's first row of the round
+                const long long n = n0 + lane;
+                const bool mine = n < total;
+                ccdc_stream_row R = {0, 0, 0};
+                long long tile0 = 0;
+                int x = 0;
+                if (mine) {
+                    while (n >= first + nrows) {    // on to the item that holds row n (items without rows are skipped)
+                        first += nrows;
+                        ++it;
+                        I = item_of(p, it);
+                        nrows = item_rows(p, I);
+                        if (nrows) {
+                            C = p.cells[I.cell];
+                            row_base = C.row0 + p.chunk_row0[I.cell * (p.nchunk + 1) + I.chunk];
+                        }
                     }
+                    x = (int)(n - first);
+                    R = p.rows[row_base + x];
+                    tile0 = I.tile * TILE_WORDS;
                 }
-                const int x = (int)(n - first);
-                const ccdc_stream_row R = p.rows[row_base + x];
-                const long long tile0 = I.tile * TILE_WORDS;
-                const int valid = (int)max(0LL, min((long long)TILE_WORDS, (long long)R.vl - tile0));
+                const int valid = mine ? (int)max(0LL, min((long long)TILE_WORDS, (long long)R.vl - tile0)) : 0;
                 const uint32_t *src = ((R.flags & CCDC_SROW_FROM_CODED) ? p.coded : p.part[C.src_node]) + R.off + tile0;
                 const uintptr_t g = reinterpret_cast<uintptr_t>(src);
                 const unsigned shift = valid > 0 ? (unsigned)(g & 15u) : 0u;
-                if (use > 0) ok = mbar_wait(&sh->empty[st], (use - 1) & 1u, abort_flag);
-                if (!ok) break;
+                if (round > 0) {                    // all of the warp's stages released by the consumers?
+                    bool all = false;
+                    for (int i = 0; i < WAIT_LIMIT && !all; ++i) {
+                        const bool freed = !mine || mbar_try(&sh->empty[st], (round - 1) & 1u);
+                        all = __all_sync(mask, freed);
+                        if (!all && (i & 15) == 15 && *abort_flag) break;
+                    }
+                    ok = all;
+                }
+                if (!ok || !mine) continue;         // (ok is the same in every lane: the loop ends for all of them)
                 unsigned desc = (unsigned)valid | ((unsigned)R.flags << 16) | (shift ? H_SHIFT : 0u);
                 if (x == nrows - 1) {
                     desc |= H_END_ITEM;
@@ -246,19 +268,21 @@ k_stream(const __grid_constant__ StreamParams p) {
                 }
             }
             if (!ok) {
-                *abort_flag = 1;
-                atomicExch(p.status, 1);
-                // let the copy already issued land before the block's shared memory is given up
-                if (use > 0) mbar_wait_plain(&sh->full[st], (use - 1) & 1u);
+                if (lane == 0) { *abort_flag = 1; atomicExch(p.status, 1); }
+                // let the copy this lane may have in flight (filled in the round before the one that gave up) land
+                // before the block's shared memory is given up
+                if (round >= 2) mbar_wait_plain(&sh->full[st], (round - 2) & 1u);
             }
         }
         return;
     }
 
-    // ---------------- consumers
-    uint32_t S[VECS][2], X[VECS][2], A[VECS][2];
+    // ---------------- consumers: thread t owns words 4t .. 4t+3 of every 512-word slice of the tile
+    uint32_t S[VECS][4], X[VECS][4], A[VECS][4];
 #pragma unroll
-    for (int v = 0; v < VECS; ++v) S[v][0] = S[v][1] = X[v][0] = X[v][1] = A[v][0] = A[v][1] = 0u;
+    for (int v = 0; v < VECS; ++v)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) S[v][c] = X[v][c] = A[v][c] = 0u;
     int st = 0;
     unsigned phase = 0;
     for (long long n = 0; n < total; ++n, st = st + 1 == p.nstage ? 0 : st + 1, phase ^= st == 0 ? 1u : 0u) {
@@ -269,15 +293,24 @@ k_stream(const __grid_constant__ StreamParams p) {
         const unsigned d = sh->head[st].desc;
         const int valid = (int)(d & 0xffffu);
         const unsigned f = (d >> 16) & 0xffu;
-        const uint32_t *words = reinterpret_cast<const uint32_t *>(ring + (size_t)st * p.stage_bytes + ((d & H_SHIFT) ? 8 : 0));
-        uint32_t in[VECS][2];
+        const bool shifted = (d & H_SHIFT) != 0;        // the row starts 8 bytes into the stage: two 64-bit loads per vector
+        const uint32_t *words = reinterpret_cast<const uint32_t *>(ring + (size_t)st * p.stage_bytes + (shifted ? 8 : 0));
+        uint32_t in[VECS][4];
 #pragma unroll
         for (int v = 0; v < VECS; ++v) {
-            const int w = (v * CONSUMERS + (int)threadIdx.x) * 2;
-            in[v][0] = in[v][1] = 0u;
-            if (w < valid) {            // valid is even: a vector is whole or absent
+            const int w = (v * CONSUMERS + (int)threadIdx.x) * 4;
+            const int left = valid - w;                 // even: 4 or more, 2, or none
+            in[v][0] = in[v][1] = in[v][2] = in[v][3] = 0u;
+            if (left >= 4 && !shifted) {
+                const uint4 q = *reinterpret_cast<const uint4 *>(words + w);
+                in[v][0] = q.x; in[v][1] = q.y; in[v][2] = q.z; in[v][3] = q.w;
+            } else if (left >= 2) {
                 const uint2 q = *reinterpret_cast<const uint2 *>(words + w);
                 in[v][0] = q.x; in[v][1] = q.y;
+                if (left >= 4) {
+                    const uint2 q2 = *reinterpret_cast<const uint2 *>(words + w + 2);
+                    in[v][2] = q2.x; in[v][3] = q2.y;
+                }
             }
         }
         const bool end = (d & H_END_ITEM) != 0;
@@ -288,39 +321,60 @@ k_stream(const __grid_constant__ StreamParams p) {
         // the row's role is the same for every word: branch once, not per vector
         if (f & CCDC_SROW_CODED) {
 #pragma unroll
-            for (int v = 0; v < VECS; ++v) { X[v][0] = in[v][0]; X[v][1] = in[v][1]; }
+            for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) X[v][c] = in[v][c];
         } else {
             if (f & CCDC_SROW_FIRST_FILE) {
 #pragma unroll
-                for (int v = 0; v < VECS; ++v) { S[v][0] = in[v][0]; S[v][1] = in[v][1]; }
+                for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) S[v][c] = in[v][c];
             } else {
 #pragma unroll
-                for (int v = 0; v < VECS; ++v) { S[v][0] = add_word<F32>(S[v][0], in[v][0]); S[v][1] = add_word<F32>(S[v][1], in[v][1]); }
+                for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) S[v][c] = add_word<F32>(S[v][c], in[v][c]);
             }
             if (f & CCDC_SROW_LAST_FILE) {
                 if (f & CCDC_SROW_FIRST_OP) {
 #pragma unroll
-                    for (int v = 0; v < VECS; ++v) { X[v][0] = S[v][0]; X[v][1] = S[v][1]; }
+                    for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) X[v][c] = S[v][c];
                 } else {
 #pragma unroll
-                    for (int v = 0; v < VECS; ++v) { X[v][0] ^= S[v][0]; X[v][1] ^= S[v][1]; }
+                    for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) X[v][c] ^= S[v][c];
                 }
             }
         }
         if ((f & (CCDC_SROW_LAST_FILE | CCDC_SROW_LAST_OP)) == (CCDC_SROW_LAST_FILE | CCDC_SROW_LAST_OP)) {
 #pragma unroll
-            for (int v = 0; v < VECS; ++v) { A[v][0] = add_word<F32>(A[v][0], X[v][0]); A[v][1] = add_word<F32>(A[v][1], X[v][1]); }
+            for (int v = 0; v < VECS; ++v)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) A[v][c] = add_word<F32>(A[v][c], X[v][c]);
         }
         if (end) {
             // The item's tile is complete.  Encode: the coded words are X itself (adding the one batch to zero
-            // would turn -0.0 into +0.0).  Decode: the sum over the batches.
+            // would turn -0.0 into +0.0).  Decode: the sum over the batches.  The output tile may itself start
+            // 8 bytes off a 16-byte boundary (segments of 4k+2 words): 64-bit stores then.
             uint32_t *dst = p.out + dst_off;
+            const bool dst16 = (reinterpret_cast<uintptr_t>(dst) & 15u) == 0;
 #pragma unroll
             for (int v = 0; v < VECS; ++v) {
-                const int w = (v * CONSUMERS + (int)threadIdx.x) * 2;
-                if (w < out_valid)
-                    *reinterpret_cast<uint2 *>(dst + w) = p.decode ? make_uint2(A[v][0], A[v][1]) : make_uint2(X[v][0], X[v][1]);
-                A[v][0] = A[v][1] = 0u;
+                const int w = (v * CONSUMERS + (int)threadIdx.x) * 4;
+                const int left = out_valid - w;
+                uint32_t o[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) { o[c] = p.decode ? A[v][c] : X[v][c]; A[v][c] = 0u; }
+                if (left >= 4 && dst16) {
+                    *reinterpret_cast<uint4 *>(dst + w) = make_uint4(o[0], o[1], o[2], o[3]);
+                } else if (left >= 2) {
+                    *reinterpret_cast<uint2 *>(dst + w) = make_uint2(o[0], o[1]);
+                    if (left >= 4) *reinterpret_cast<uint2 *>(dst + w + 2) = make_uint2(o[2], o[3]);
+                }
             }
         }
     }
@@ -347,7 +401,7 @@ void ring_shape(const ccdc_plan_s &P, int *nstage, int *stage_bytes, size_t *sme
     *stage_bytes = (int)((tile * 4 + 16 + 127) / 128 * 128);
     const size_t fixed = (sizeof(Shared) + 127) / 128 * 128;
     const long long n = (long long)(((size_t)CCDC_STREAM_SMEM_BYTES - fixed) / *stage_bytes);
-    *nstage = (int)std::max(2LL, std::min<long long>(n, MAX_STAGES));
+    *nstage = (int)std::max<long long>(PRODUCERS, std::min<long long>(n, MAX_STAGES) / PRODUCERS * PRODUCERS);
     *smem = fixed + (size_t)*nstage * *stage_bytes;
 }
 
