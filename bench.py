@@ -282,7 +282,7 @@ def run_reference(args, w):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32" if w.dtype == "float32" else "i32",
         "data": "synthetic", "config": {"workload": w.name, "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
                          "sample_reason": SAMPLE_REASON if B < w.B else "full size", **host_cpu()},
@@ -597,7 +597,7 @@ def run_ours(args, w):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "strong" if (sharded or value_sharded) else "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32" if w.dtype == "float32" else "i32", "data": "synthetic",
         "config": {"workload": w.name, "parallelism": f"nodes sharded over {world} GPUs, {wire['exchange']}" if sharded
                    else f"one job, every segment cut into {world} sub-ranges, one per GPU, no exchange (B={full_B})" if value_sharded
                    else f"{world} independent job(s), one per GPU", "K": w.K, "r": w.r, "N": w.N, "Q": w.Q, "B": w.B,

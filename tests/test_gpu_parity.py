@@ -676,3 +676,42 @@ def test_back_to_back_steps_on_the_same_buffers(ccdc, K, r, N, Q, B, chunks):
         assert np.array_equal(bits(c).reshape(-1, sp)[:, :s], refs[which][0].reshape(-1, s))
         assert np.array_equal(o_.cpu().numpy().reshape(refs[which][1].shape), refs[which][1])
     plan.shuffle_status()
+
+
+def test_jobs20_structure_short_values(ccdc):
+    """The paper's own setting at the benchmark's scale of nodes -- K=20, r=2, J = C(20,3) = 1140 jobs of
+    21 files, 7 per batch, stage 1 and 17 stage-2 rounds per subset -- with short values: every coded
+    word, packet and output against the oracle, and the load of Theorem 1."""
+    from fractions import Fraction
+
+    w = CONFIGS["jobs20"].scaled(96)
+    plan = run_case(ccdc, w.K, w.r, w.N, w.Q, w.B, w.dtype, jobs=True, std=w.std)
+    assert plan.J == 1140 and plan.files_per_batch == 7 and plan.num_groups == 1140 * 18
+    assert Fraction(plan.coded_bits, plan.J * w.Q * 32 * w.B) == Fraction(27, 20)       # (1-mu)(mu K+1)/(mu K) = 1.35
+    assert "files=4" in ccdc.last_decode_kernel()
+
+
+def test_bench_line_contract(ccdc):
+    """`python bench.py --workload cfg1`: one JSON line with every key the measurement contract names."""
+    import json
+    import subprocess
+    import sys
+    from pathlib import Path
+
+    root = Path(__file__).resolve().parent.parent
+    res = subprocess.run([sys.executable, str(root / "bench.py"), "--workload", "cfg1", "--steps", "5", "--warmup", "3"],
+                         capture_output=True, text=True, timeout=900, cwd=str(root))
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "roofline", "cpu_baseline", "e2e", "gpu_launches", "clocks"):
+        assert key in d, key
+    assert d["n_gpus"] == 1 and d["steps"] == 5 and d["warmup"] == 3 and d["dtype"] == "i32"
+    assert d["config"]["workload"] == "cfg1" and d["vs_baseline"] is None and d["value"] > 0
+    for key in ("bound", "achieved", "peak", "unit", "frac", "frac_nominal", "traffic", "algorithmic_gbs"):
+        assert key in d["roofline"], key
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] == 1 and d["cpu_baseline"]["value"] > 0
+    assert d["e2e"]["h2d_bytes_per_step"] == 12 * 4 * 256 * 4 and d["e2e"]["d2h_bytes_per_step"] == 4 * 256 * 4
+    assert d["gpu_launches"] >= 2 * 5
