@@ -11,9 +11,10 @@
 // of the job's batches for the decode).  The source rows of all its items form
 // ONE sequence.  Two producer warps, each owning half of a ring of
 // shared-memory stages (one lane per stage, the lanes in lockstep), stream that
-// sequence in with bulk asynchronous copies, running ahead across item boundaries, so tens of KiB are in flight per block
-// all the time and none of them in registers; 128 consumer threads fold the
-// rows, in the order the scheme fixes, into three registers per word:
+// sequence in with bulk asynchronous copies, running ahead across item
+// boundaries, so tens of KiB are in flight per block all the time and none of
+// them in registers; 128 consumer threads fold the rows, in the order the
+// scheme fixes, into three registers per word:
 //     S  running sum over the files of the current operand   (pre-combining)
 //     X  XOR over the operands of the current batch           (coding / decoding)
 //     A  sum over the batches                                  (Eq. (1))
