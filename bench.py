@@ -49,6 +49,8 @@ NCU_TRAFFIC = {
              1024, 2256828424.0, "profiles/ncu_jobs20_small.md"),
     "cfg2": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
              4096, 145249792.0, "profiles/ncu_cfg2_full.md"),
+    "compression:cfg4": ("k_gather(combine)+k_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
+             128000, 2144084880.0, "profiles/ncu_compression_small.md"),
     "cfg5": ("k_map", "a7427ce9fd62495f5562f015e6406acaf19ca4a6b7c5b8c4ef81d0fa3406c4a7",
              1024, 2826514184.0, "profiles/k_map_cluster_cfg5.md"),
 }
