@@ -678,6 +678,56 @@ def test_back_to_back_steps_on_the_same_buffers(ccdc, K, r, N, Q, B, chunks):
     plan.shuffle_status()
 
 
+def random_shapes(seed, count):
+    """`count` parameter sets of the scheme drawn from a seeded generator: K up to 12, every r, 1 to 9 files
+    per batch, Q/K up to 3, value lengths from 1 to 24 000 words, one job or the J-job setting, both
+    dtypes; some with the bulk-copy kernels, some with a drawn launch shape of the fused decode."""
+    import random
+
+    rng = random.Random(seed)
+    while count > 0:
+        jobs = rng.random() < 0.2
+        K = rng.randint(3, 6 if jobs else 12)
+        r = rng.randint(1, K - 1)
+        if jobs:
+            N = rng.randint(1, 4) * (r + 1)
+            if comb(K, r + 1) > 60 or N < K:
+                continue
+        else:
+            if comb(K, r) > 500:
+                continue
+            N = rng.choice([1, 1, 2, 3, 4, 5, 7, 9]) * comb(K, r)
+        Q = K * rng.choice([1, 1, 1, 2, 3])
+        kind = rng.random()
+        B = rng.randint(1, 40) if kind < 0.3 else rng.randint(41, 3000) if kind < 0.7 else rng.randint(3000, 24000)
+        if (comb(K, r + 1) if jobs else 1) * N * Q * B > 12_000_000:
+            continue
+        dtype = rng.choice(["int32", "float32"])
+        family = 1 if rng.random() < 0.3 and bulk_copy_family_serves(K, r, N, Q, B) else None
+        shape = (rng.random() < 0.5, rng.random() < 0.5, rng.randint(1, 16))    # override?, short blocks?, chunks
+        yield K, r, N, Q, B, dtype, jobs, family, shape
+        count -= 1
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13, 14])
+def test_random_shapes_match_oracle(ccdc, seed):
+    """Thirty drawn parameter sets per seed, each through the stepwise and the fused path against the oracle."""
+    for case, (K, r, N, Q, B, dtype, jobs, family, (override, short, chunks)) in enumerate(random_shapes(seed, 30)):
+        tune = None
+        if family is None and override:
+            probe = ccdc.Plan(K, r, N, Q, B, dtype, jobs=jobs)
+            threads = probe.decode_threads if probe.decode_threads == 128 else (1024 if short else 512)
+            try:
+                probe.tune_decode(threads, chunks)
+                tune = (threads, chunks)
+            except ccdc.CcdcError as e:         # more chunks than terms in the batch loop
+                assert e.status == ccdc.EINVAL
+        try:
+            run_case(ccdc, K, r, N, Q, B, dtype, jobs=jobs, seed=seed * 100 + case, tune=tune, family=family)
+        except AssertionError as e:
+            raise AssertionError(f"{(K, r, N, Q, B, dtype, jobs, family, tune)}: {e}") from e
+
+
 def test_jobs20_structure_short_values(ccdc):
     """The paper's own setting at the benchmark's scale of nodes -- K=20, r=2, J = C(20,3) = 1140 jobs of
     21 files, 7 per batch, stage 1 and 17 stage-2 rounds per subset -- with short values: every coded
