@@ -728,6 +728,52 @@ def test_random_shapes_match_oracle(ccdc, seed):
             raise AssertionError(f"{(K, r, N, Q, B, dtype, jobs, family, tune)}: {e}") from e
 
 
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_shapes_through_the_other_entry_points(ccdc, seed):
+    """Twenty-five drawn parameter sets per seed through the compression-only comparator, the node-sharded
+    plans (all ranks on this GPU, one after the other) and the two entries that start from host memory."""
+    import random
+
+    rng = random.Random(seed)
+    done = 0
+    while done < 25:
+        what = rng.choice(["comparator", "node shards", "host files", "host buffers"])
+        dtype = rng.choice(["int32", "float32"])
+        K = rng.randint(3, 10)
+        r = rng.randint(1, K - 1)
+        Q = K * rng.choice([1, 1, 2])
+        kind = rng.random()
+        B = rng.randint(1, 40) if kind < 0.3 else rng.randint(41, 3000) if kind < 0.7 else rng.randint(3000, 12000)
+        jobs = what in ("node shards", "host files") and rng.random() < 0.3
+        if what == "comparator":
+            N = rng.randint(K, 60)
+            if (r * N) % K or N - (-(-K // r) - 1) * (r * N // K) < 1:
+                continue
+        elif jobs:
+            N = rng.randint(1, 3) * (r + 1)
+            if K > 6 or comb(K, r + 1) > 40 or N < K:
+                continue
+        else:
+            if comb(K, r) > 260:
+                continue
+            N = rng.choice([1, 2, 3, 4]) * comb(K, r)
+        if (comb(K, r + 1) if jobs else 1) * N * Q * B > 6_000_000:
+            continue
+        try:
+            if what == "comparator":
+                test_compression_only_matches_oracle(ccdc, K, r, N, Q, B, dtype)
+            elif what == "node shards":
+                worlds = [w for w in range(2, K + 1) if K % w == 0]
+                test_node_sharded_ranks_emulated_on_one_gpu(ccdc, K, r, N, Q, B, rng.choice(worlds), jobs, dtype)
+            elif what == "host files":
+                test_shuffle_from_host_files(ccdc, K, r, N, Q, B, jobs, dtype)
+            else:
+                test_shuffle_from_host_buffers(ccdc, K, r, N, Q, B, dtype)
+        except AssertionError as e:
+            raise AssertionError(f"{what} {(K, r, N, Q, B, dtype, jobs)}: {e}") from e
+        done += 1
+
+
 def test_jobs20_structure_short_values(ccdc):
     """The paper's own setting at the benchmark's scale of nodes -- K=20, r=2, J = C(20,3) = 1140 jobs of
     21 files, 7 per batch, stage 1 and 17 stage-2 rounds per subset -- with short values: every coded
