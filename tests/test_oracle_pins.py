@@ -577,3 +577,48 @@ def test_every_step_acts_word_by_word_along_a_segment(mode, dtype):
         want = out.reshape(full.J * K, per * B)[:, pos].reshape(got.shape)
         assert np.array_equal(got.view(np.uint32), np.ascontiguousarray(want).view(np.uint32))
         assert part.coded_bits * s == full.coded_bits * w
+
+
+# ---------------------------------------------- drawn parameter sets, both settings
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_drawn_parameter_sets_obey_the_definition_and_the_load(seed):
+    """Forty parameter sets per seed (K up to 8, every r, several files per batch, Q/K up to 3, value lengths
+    that r does or does not divide; one job or J = C(K, r+1) jobs): every output is the wrapped sum of
+    Eq. (1) written with numpy, every receiver decodes (the shuffle reports nothing), the multicast bits are
+    rounds x (r+1) packets x 32 s, and, where r divides the packet, the J-job load is Theorem 1's."""
+    import random
+
+    rng = random.Random(seed)
+    done = 0
+    while done < 40:
+        paper = rng.random() < 0.4
+        K = rng.randint(2, 6 if paper else 8)
+        r = rng.randint(1, K - 1)
+        per = rng.choice([1, 1, 2, 3])
+        B = rng.randint(1, 24)
+        if paper:
+            N = rng.randint(1, 3) * (r + 1)
+            if N < K or comb(K, r + 1) > 40:
+                continue
+            J, rounds, b = comb(K, r + 1), comb(K, r + 1) * (K - r), N // (r + 1)
+        else:
+            b = rng.randint(1, 4)
+            N = b * comb(K, r)
+            if N < K:
+                continue
+            J, rounds = 1, comb(K, r + 1)
+        Q = per * K
+        v = values_numpy(J * N, Q, B, "int32", seed=seed * 1000 + done)
+        o = Oracle(K, r, N, Q, B, "int32", mode="paper" if paper else "single")
+        o.load_values(v)
+        assert o.shuffle_status() == 0, (K, r, N, Q, B, paper)
+        out = o.reduce().reshape(J, Q, B)
+        expect = (v.reshape(J, N, Q, B).astype(np.int64).sum(axis=1) & 0xFFFFFFFF).astype(np.uint32).view(np.int32)
+        assert np.array_equal(out, expect), (K, r, N, Q, B, paper)
+        s = -(-(per * B) // r)
+        assert (o.J, o.nround, o.b, o.s) == (J, rounds, b, s)
+        assert o.coded_bits == rounds * (r + 1) * 32 * s
+        if paper and (per * B) % r == 0:
+            mu = Fraction(r, K)
+            assert Fraction(o.coded_bits, J * Q * 32 * B) == (1 - mu) * (mu * K + 1) / (mu * K)
+        done += 1
