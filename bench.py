@@ -41,16 +41,16 @@ UNIT = "GB/s"
 # measured on (hash over the files listed); otherwise the line reports null.
 NCU_TRAFFIC = {
     # workload: (kernel, sources sha256, value elements of the capture, DRAM bytes of that launch, profile)
-    "cfg4": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
-             128000, 3542451624.0, "profiles/ncu_cfg4_small.md"),
-    "cfg3": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
-             8208, 3114471640.0, "profiles/ncu_cfg3_small.md"),
-    "jobs20": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
-             1024, 2256828424.0, "profiles/ncu_jobs20_small.md"),
-    "cfg2": ("k_decode_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
-             4096, 145249792.0, "profiles/ncu_cfg2_full.md"),
-    "compression:cfg4": ("k_gather(combine)+k_reduce", "a27b267fe5eac5c439582d0e2fd7ebd2d5888477b719b9c2c19bdee764921d90",
-             128000, 2144084880.0, "profiles/ncu_compression_small.md"),
+    "cfg4": ("k_decode_reduce", "60a405a7a0446a11b9ca011cd2614cde98348f8b6d7edb13cf7d7d80c5b447b3",
+             128000, 3541666520.0, "profiles/ncu_cfg4_small.md"),
+    "cfg3": ("k_decode_reduce", "60a405a7a0446a11b9ca011cd2614cde98348f8b6d7edb13cf7d7d80c5b447b3",
+             8208, 3113737120.0, "profiles/ncu_cfg3_small.md"),
+    "jobs20": ("k_decode_reduce", "60a405a7a0446a11b9ca011cd2614cde98348f8b6d7edb13cf7d7d80c5b447b3",
+             1024, 2256910400.0, "profiles/ncu_jobs20_small.md"),
+    "cfg2": ("k_decode_reduce", "60a405a7a0446a11b9ca011cd2614cde98348f8b6d7edb13cf7d7d80c5b447b3",
+             4096, 144492544.0, "profiles/ncu_cfg2_full.md"),
+    "compression:cfg4": ("k_gather(combine)+k_reduce", "60a405a7a0446a11b9ca011cd2614cde98348f8b6d7edb13cf7d7d80c5b447b3",
+             128000, 2141599280.0, "profiles/ncu_compression_small.md"),
     "cfg5": ("k_map", "a7427ce9fd62495f5562f015e6406acaf19ca4a6b7c5b8c4ef81d0fa3406c4a7",
              1024, 2826514184.0, "profiles/k_map_cluster_cfg5.md"),
 }

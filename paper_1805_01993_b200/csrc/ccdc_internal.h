@@ -18,6 +18,9 @@
 #ifndef CCDC_DECODE_THREADS_FILES
 #define CCDC_DECODE_THREADS_FILES 128   // used when several files of a batch are loaded together
 #endif
+#ifndef CCDC_DECODE_BLOCKS_FILES         // blocks of that kernel resident per SM, by vector width (planner and kernel agree)
+#define CCDC_DECODE_BLOCKS_FILES(vec) ((vec) <= 2 ? 7 : 6)
+#endif
 #ifndef CCDC_DECODE_FILES_MAX
 #define CCDC_DECODE_FILES_MAX 4         // most files of a batch loaded together (4, 2; 1 = batch-by-batch kernel)
 #endif

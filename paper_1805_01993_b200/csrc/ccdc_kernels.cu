@@ -484,9 +484,10 @@ struct DecodeParams {
 // Blocks per SM the register allocation is held to (the compiler's own choice moves with every
 // change to the kernel, and the streaming rate follows the resident threads): blocks of 512 threads
 // with little in flight per thread at 3 per SM (40 registers), with more at 2 (64); several files in
-// flight: up to 80 registers.
+// flight: 6 blocks of 128 threads (80 registers) with 128-bit accesses, 7 (72 registers, which those
+// kernels fill without spilling) with narrower ones.
 constexpr int decode_min_blocks(int vec, int nt, int r1s, int g) {
-    if (g > 1) return nt <= 128 ? 6 : nt <= 256 ? 3 : 2;
+    if (g > 1) return nt <= 128 ? CCDC_DECODE_BLOCKS_FILES(vec) : nt <= 256 ? 3 : 2;
     if (nt >= 1024) return 1;
     if (r1s < 0) return vec <= 2 ? 3 : 2;
     return (1 + r1s) * vec * CCDC_DECODE_DEPTH <= 16 ? 3 : 2;

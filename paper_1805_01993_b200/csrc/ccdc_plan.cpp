@@ -122,6 +122,7 @@ void choose_split(ccdc_plan_s &P, long long nout) {
     // blocks resident per SM at the registers these kernels take
     auto resident = [&](int threads) {
         if (P.family == 1) return (long long)P.sm_count * 3;       // bulk-copy pipeline: shared memory for three blocks
+        if (threads == CCDC_DECODE_THREADS_FILES && group > 1) return (long long)P.sm_count * CCDC_DECODE_BLOCKS_FILES(P.vec);
         return (long long)P.sm_count * (threads >= 1024 ? 1 : threads >= 512 ? 3 : 768 / threads);
     };
     // enough thread blocks to fill the GPU (8 per SM) while a block still walks a fair number of batches
