@@ -195,6 +195,35 @@ print("register variant ok")
 """
 
 
+@pytest.mark.parametrize("seed", [31, 32])
+def test_drawn_map_jobs(ccdc, seed):
+    """Ten drawn jobs per seed inside the shapes the Map accepts (rows a multiple of 16, d a multiple of
+    512): K up to 8, every r, up to 3 files per batch, Q/K up to 2; Map values, replicas, coded rows and
+    outputs as in run_job.  Both Map kernels are reached."""
+    import random
+    from math import comb
+
+    rng = random.Random(seed)
+    done, kernels = 0, set()
+    while done < 10:
+        K = rng.randint(3, 8)
+        r = rng.randint(1, K - 1)
+        N = rng.choice([1, 1, 2, 3]) * comb(K, r)
+        Q = K * rng.choice([1, 1, 2])
+        d = 512 * rng.choice([1, 2, 3, 4, 4, 5, 8, 8, 12, 16, 16, 32, 32])
+        rows = 16 * rng.choice([1, 2, 2, 3, 4, 5, 8, 10, 16, 32])
+        if comb(K, r) > 60 or N < K or d % Q or N * rows * d > 40_000_000:
+            continue
+        try:
+            worst = run_job(ccdc, K, r, N, Q, d // Q, rows=rows, seed=seed * 100 + done)
+        except AssertionError as e:
+            raise AssertionError(f"{(K, r, N, Q, d // Q, rows)}: {e}") from e
+        assert worst < 1e-5
+        kernels.add(ccdc.map_last_kernel())
+        done += 1
+    assert kernels == {"k_map", "k_map_cluster"}
+
+
 def test_register_kernel_on_cluster_shapes(ccdc, tmp_path):
     """The register kernel is the fallback for devices that cannot run the cluster kernel: built
     with the cluster kernel switched off, it is held to the same parity on the shapes the cluster
